@@ -1,0 +1,176 @@
+/*
+ * sparsed.h - C ABI of the SparseD attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the attention hot path of SparseD (sparse attention for
+ * diffusion language models): dense bidirectional attention for the early denoising
+ * steps, a one-off per-head block-pattern selection at the switch step, and
+ * block-sparse attention that reuses the pattern for all later steps (Algorithm 1).
+ *
+ * Conventions for every entry point
+ *  - Pointers marked "device" are CUDA device pointers owned by the caller; the
+ *    library never allocates or frees device memory and keeps no reference to caller
+ *    buffers after a call returns. Pointers marked "host" are ordinary host pointers.
+ *  - Tensors: Q and O are [batch, heads_q, seq_len, head_dim], K and V are
+ *    [batch, heads_kv, seq_len, head_dim], bf16, head_dim contiguous. Strides for
+ *    (batch, head, token) are given in elements; all-zero strides mean "contiguous".
+ *    Base pointers must be 16-byte aligned and every stride a multiple of 8 elements.
+ *  - Grouped-query attention: query head h reads key/value head h / (heads_q / heads_kv).
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *    stream) and return without synchronising. Argument problems are detected on the
+ *    host before anything is launched and reported through the return code.
+ *  - Every call takes a workspace `ws` (device) of at least
+ *    sparsed_workspace_bytes(op, ...) bytes. Its first SPARSED_STATUS_BYTES bytes hold the
+ *    device status word and must be zero before the first call (sparsed_workspace_init).
+ *    Kernels never trap or spin forever: a wait that runs out records itself in the
+ *    status word, which sparsed_last_device_status reads back.
+ *  - Results are deterministic: the same inputs give bitwise the same outputs.
+ */
+#ifndef SPARSED_H_
+#define SPARSED_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum sparsed_status {
+  SPARSED_OK = 0,
+  SPARSED_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, heads_q % heads_kv != 0, ... */
+  SPARSED_ERR_UNSUPPORTED = 2,    /* head_dim != 128, block_size not in {64,128}, too many blocks */
+  SPARSED_ERR_ALIGNMENT = 3,      /* seq_len or prefill_len not a multiple of block_size; pointer/stride alignment */
+  SPARSED_ERR_WORKSPACE = 4,      /* workspace missing or too small */
+  SPARSED_ERR_PATTERN = 5,        /* pattern arrays missing, too small, or inconsistent with the shape */
+  SPARSED_ERR_ARCH = 6,           /* current device is not compute capability 10.x */
+  SPARSED_ERR_CUDA = 7,           /* a CUDA call failed; see sparsed_last_cuda_error() */
+  SPARSED_ERR_DEVICE_TIMEOUT = 8  /* a bounded device-side wait ran out (from the status word) */
+} sparsed_status;
+
+#define SPARSED_STATUS_BYTES 256
+
+/* Operation ids for sparsed_workspace_bytes. */
+#define SPARSED_OP_ATTN_FULL 0
+#define SPARSED_OP_SELECT_PATTERN 1
+#define SPARSED_OP_SELECT_FROM_SCORES 2
+#define SPARSED_OP_ATTN_SPARSE 3
+#define SPARSED_OP_PATTERN_VALIDATE 4
+
+/* Schedule modes returned by sparsed_schedule_mode. */
+#define SPARSED_MODE_FULL 0
+#define SPARSED_MODE_FULL_AND_SELECT 1
+#define SPARSED_MODE_SPARSE 2
+
+typedef struct sparsed_shape {
+  int32_t batch, heads_q, heads_kv, seq_len, head_dim;
+  int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3]; /* elements: batch, head, token */
+  float softmax_scale;                                            /* 0 => 1/sqrt(head_dim) */
+} sparsed_shape;
+
+typedef struct sparsed_select_params {
+  int32_t block_size;  /* 64 or 128 */
+  int32_t prefill_len; /* p of Eq. 6: keys [0,p) are prefill, [p,seq_len) generation; multiple of block_size */
+  double keep_ratio;   /* rho in (0,1] */
+  int32_t rounding;    /* 0: kept = ceil(rho * blocks in region) (default), 1: floor; at least 1 */
+} sparsed_select_params;
+
+/* Block pattern of Eq. 4 as CSR lists: row r = (b*heads_q + h)*num_blocks + query_block;
+ * col_idx[row_ptr[r] .. row_ptr[r+1]) are the kept key blocks, strictly ascending. */
+typedef struct sparsed_pattern {
+  int32_t *row_ptr;     /* device, batch*heads_q*num_blocks + 1 entries */
+  int32_t *col_idx;     /* device, col_capacity entries */
+  int64_t col_capacity; /* entries available in col_idx */
+  int64_t nnz;          /* set by the selection calls: entries used */
+  int32_t block_size, num_blocks, batch, heads_q; /* set by the selection calls */
+} sparsed_pattern;
+
+/*
+ * Dense bidirectional attention, O = softmax(Q K^T / sqrt(d)) V with no mask (Eq. 1 and
+ * the "A(Q,K) V" of Section 3.1; the full-attention branch of Algorithm 1).
+ * q,k,v,o: device bf16. lse_or_null: device fp32 [batch, heads_q, seq_len] receiving the
+ * natural-log sum of exponentials of each query row's scaled logits, or NULL.
+ * Any seq_len >= 1 is accepted. Errors: INVALID_ARG, UNSUPPORTED (head_dim != 128),
+ * ALIGNMENT, WORKSPACE, ARCH, CUDA.
+ */
+sparsed_status sparsed_attn_full(const sparsed_shape *shape, const void *q, const void *k, const void *v,
+                                 void *o, float *lse_or_null, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Pattern selection at the switch step ("Isolated Selection", Eq. 5 and Eq. 6, the inner
+ * loop of Algorithm 1): A' = avgpool(softmax(Q K^T / sqrt(d)), block_size) is computed one
+ * query block at a time without materialising the l x l matrix; for each head and query
+ * block the top-rho% key blocks are chosen separately among prefill and generation blocks,
+ * ranked by A' (fp32), ties to the lower block index, and written as ascending CSR lists.
+ * lse_or_null: the LSE written by sparsed_attn_full for the same Q,K (saves a pass), or NULL.
+ * scores_out_or_null: device fp32 [batch, heads_q, nb, nb] receiving A', or NULL (then the
+ * workspace holds it). `out`: host struct; its row_ptr/col_idx/col_capacity are inputs, the
+ * other fields are filled in. Requires seq_len % block_size == 0 and
+ * prefill_len % block_size == 0. Errors: as above plus PATTERN (capacity too small).
+ */
+sparsed_status sparsed_select_pattern(const sparsed_shape *shape, const sparsed_select_params *params,
+                                      const void *q, const void *k, const float *lse_or_null,
+                                      sparsed_pattern *out, float *scores_out_or_null, void *ws,
+                                      size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The ranking half of the selection alone (Eq. 5 / Eq. 6 applied to a given A'):
+ * scores: device fp32 [batch, heads_q, num_blocks, num_blocks]. NaN scores rank lowest.
+ */
+sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, const float *scores,
+                                          int32_t batch, int32_t heads_q, int32_t num_blocks,
+                                          sparsed_pattern *out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Block-sparse attention, O = softmax((Q K^T + M_S) / sqrt(d)) V with M_S the 0 / -inf block
+ * mask given by `pattern` (Eq. 3 and Eq. 4; the "Sparse Reusing" branch of Algorithm 1).
+ * Accepts any CSR whose rows are ascending and in range (not only selected ones); a query
+ * block with an empty list gets zeros. Requires seq_len == pattern->num_blocks *
+ * pattern->block_size. Errors: as above plus PATTERN.
+ */
+sparsed_status sparsed_attn_sparse(const sparsed_shape *shape, const sparsed_pattern *pattern, const void *q,
+                                   const void *k, const void *v, void *o, void *ws, size_t ws_bytes,
+                                   void *cuda_stream);
+
+/*
+ * Step schedule ("Skipping Sparse", the outer branch of Algorithm 1). Steps are 1-based.
+ * The switch step is s = clamp(floor(total_steps * skip), 1, total_steps); steps before s
+ * are FULL, step s is FULL_AND_SELECT (full attention, then select), later steps SPARSE.
+ * Host only. sparsed_schedule_mode returns a SPARSED_MODE_* value or -1 on bad arguments;
+ * sparsed_switch_step returns s or -1.
+ */
+int32_t sparsed_schedule_mode(int32_t step_1based, int32_t total_steps, double skip);
+int32_t sparsed_switch_step(int32_t total_steps, double skip);
+
+/*
+ * Number of key blocks kept per query block in the prefill and generation regions
+ * (Eq. 6's "top-rho%" counted in blocks). Host only; k_pre / k_gen are host pointers.
+ */
+sparsed_status sparsed_kept_per_row(const sparsed_select_params *params, int32_t seq_len, int32_t *k_pre,
+                                    int32_t *k_gen);
+
+/* Workspace size in bytes for one SPARSED_OP_*; `shape`/`params` may be NULL where unused. Host only. */
+sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape *shape,
+                                       const sparsed_select_params *params, size_t *out_bytes);
+
+/* Zeroes the status block of a workspace (asynchronous memset on the stream). */
+sparsed_status sparsed_workspace_init(void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Checks a pattern on the device: row_ptr monotone and within capacity, every list strictly
+ * ascending and within [0, num_blocks), no empty row. Synchronises the stream. Returns
+ * SPARSED_OK or SPARSED_ERR_PATTERN. (No paper counterpart: a guard for user-built masks.)
+ */
+sparsed_status sparsed_pattern_validate(const sparsed_pattern *pattern, void *ws, size_t ws_bytes,
+                                        void *cuda_stream);
+
+/* Reads the device status word (synchronises the stream). code 0 = fine, 1 = a wait ran out;
+ * `where` identifies the wait. Returns SPARSED_ERR_DEVICE_TIMEOUT if code != 0. */
+sparsed_status sparsed_last_device_status(void *ws, void *cuda_stream, int32_t *code, int32_t *where);
+
+const char *sparsed_status_string(sparsed_status status);
+int32_t sparsed_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSED_H_ */

@@ -1,0 +1,427 @@
+// C ABI of the SparseD attention library: argument validation, tensor-map construction,
+// workspace layout and kernel dispatch. Declarations and contracts are in sparsed.h.
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/sparsed.h"
+#include "internal.h"
+
+namespace {
+
+using namespace sparsed;
+
+thread_local int32_t g_last_cuda_error = 0;
+
+sparsed_status cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int32_t>(e);
+  return SPARSED_ERR_CUDA;
+}
+
+// ---- driver entry point for tensor-map encoding (no link-time dependency on libcuda) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess) {
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+  });
+  return fn;
+}
+
+// bf16 [B,H,L,128] tensor with element strides (batch, head, token); box = 64 x rows, 128B swizzle.
+sparsed_status make_tensor_map(CUtensorMap* out, const void* base, int batch, int heads, int seq_len,
+                               const int64_t strides[3], int box_rows) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (enc == nullptr) return cuda_fail(cudaErrorNotSupported);
+  cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(seq_len), static_cast<cuuint64_t>(heads),
+                        static_cast<cuuint64_t>(batch)};
+  cuuint64_t gstrides[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
+                            static_cast<cuuint64_t>(strides[0]) * 2};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, 1};
+  cuuint32_t elem[4] = {1, 1, 1, 1};
+  CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gstrides, box, elem,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = static_cast<int32_t>(r);
+    return SPARSED_ERR_CUDA;
+  }
+  return SPARSED_OK;
+}
+
+struct Resolved {
+  int64_t q[3], k[3], v[3], o[3];
+  float scale_log2;
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void default_strides(const int64_t in[3], int heads, int seq_len, int64_t out[3]) {
+  if (in[0] == 0 && in[1] == 0 && in[2] == 0) {
+    out[2] = 128;
+    out[1] = static_cast<int64_t>(seq_len) * 128;
+    out[0] = out[1] * heads;
+  } else {
+    out[0] = in[0];
+    out[1] = in[1];
+    out[2] = in[2];
+  }
+}
+
+sparsed_status check_arch() {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  static int cached_major[64];
+  static bool cached[64] = {};
+  int major = 0;
+  if (dev >= 0 && dev < 64 && cached[dev]) {
+    major = cached_major[dev];
+  } else {
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev >= 0 && dev < 64) {
+      cached_major[dev] = major;
+      cached[dev] = true;
+    }
+  }
+  return major == 10 ? SPARSED_OK : SPARSED_ERR_ARCH;
+}
+
+sparsed_status check_shape(const sparsed_shape* s, bool need_v_o, Resolved* r) {
+  if (s == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (s->batch < 1 || s->heads_q < 1 || s->heads_kv < 1 || s->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+  if (s->heads_q % s->heads_kv != 0) return SPARSED_ERR_INVALID_ARG;
+  if (s->head_dim != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (!(s->softmax_scale >= 0.f) || !std::isfinite(s->softmax_scale)) return SPARSED_ERR_INVALID_ARG;
+  default_strides(s->q_strides, s->heads_q, s->seq_len, r->q);
+  default_strides(s->k_strides, s->heads_kv, s->seq_len, r->k);
+  default_strides(s->v_strides, s->heads_kv, s->seq_len, r->v);
+  default_strides(s->o_strides, s->heads_q, s->seq_len, r->o);
+  const int64_t* sets[4] = {r->q, r->k, r->v, r->o};
+  for (int t = 0; t < (need_v_o ? 4 : 2); ++t) {
+    for (int i = 0; i < 3; ++i) {
+      if (sets[t][i] <= 0) return SPARSED_ERR_INVALID_ARG;
+      if (sets[t][i] % 8 != 0) return SPARSED_ERR_ALIGNMENT;
+    }
+    if (sets[t][2] < 128) return SPARSED_ERR_INVALID_ARG;
+  }
+  const float scale = s->softmax_scale == 0.f ? 1.0f / std::sqrt(static_cast<float>(s->head_dim)) : s->softmax_scale;
+  r->scale_log2 = scale * 1.44269504088896341f;
+  return SPARSED_OK;
+}
+
+sparsed_status kept_counts(const sparsed_select_params* sp, int nb, int* pb, int* k_pre, int* k_gen) {
+  if (sp == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (sp->block_size != 64 && sp->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (!(sp->keep_ratio > 0.0) || !(sp->keep_ratio <= 1.0)) return SPARSED_ERR_INVALID_ARG;
+  if (sp->rounding != 0 && sp->rounding != 1) return SPARSED_ERR_INVALID_ARG;
+  if (sp->prefill_len < 0) return SPARSED_ERR_INVALID_ARG;
+  if (sp->prefill_len % sp->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  const int p_blocks = sp->prefill_len / sp->block_size;
+  if (p_blocks > nb) return SPARSED_ERR_INVALID_ARG;
+  auto kept = [&](int n) -> int {
+    if (n <= 0) return 0;
+    const double x = sp->keep_ratio * n;
+    long long kk = sp->rounding == 0 ? static_cast<long long>(std::ceil(x - 1e-6))
+                                     : static_cast<long long>(std::floor(x + 1e-6));
+    if (kk < 1) kk = 1;
+    if (kk > n) kk = n;
+    return static_cast<int>(kk);
+  };
+  *pb = p_blocks;
+  *k_pre = kept(p_blocks);
+  *k_gen = kept(nb - p_blocks);
+  return SPARSED_OK;
+}
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+sparsed_status run_topk(const float* scores, int batch, int heads_q, int nb, int block_size, int pb, int k_pre,
+                        int k_gen, sparsed_pattern* out, cudaStream_t stream) {
+  if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if (nb > 1024) return SPARSED_ERR_UNSUPPORTED;
+  const int64_t rows = static_cast<int64_t>(batch) * heads_q * nb;
+  const int64_t nnz = rows * (k_pre + k_gen);
+  if (rows >= INT32_MAX || nnz >= INT32_MAX) return SPARSED_ERR_UNSUPPORTED;
+  if (out->col_capacity < nnz) return SPARSED_ERR_PATTERN;
+  TopkParams tp;
+  tp.scores = scores;
+  tp.row_ptr = out->row_ptr;
+  tp.col_idx = out->col_idx;
+  tp.rows = static_cast<int>(rows);
+  tp.nb = nb;
+  tp.pb = pb;
+  tp.k_pre = k_pre;
+  tp.k_gen = k_gen;
+  cudaError_t e = launch_topk_csr(tp, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  out->nnz = nnz;
+  out->block_size = block_size;
+  out->num_blocks = nb;
+  out->batch = batch;
+  out->heads_q = heads_q;
+  return SPARSED_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sparsed_status_string(sparsed_status status) {
+  switch (status) {
+    case SPARSED_OK: return "ok";
+    case SPARSED_ERR_INVALID_ARG: return "invalid argument";
+    case SPARSED_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SPARSED_ERR_ALIGNMENT: return "alignment or divisibility requirement not met";
+    case SPARSED_ERR_WORKSPACE: return "workspace missing or too small";
+    case SPARSED_ERR_PATTERN: return "pattern invalid or too small";
+    case SPARSED_ERR_ARCH: return "device is not compute capability 10.x";
+    case SPARSED_ERR_CUDA: return "CUDA error";
+    case SPARSED_ERR_DEVICE_TIMEOUT: return "device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+int32_t sparsed_last_cuda_error(void) { return g_last_cuda_error; }
+
+int32_t sparsed_switch_step(int32_t total_steps, double skip) {
+  if (total_steps < 1 || !(skip >= 0.0) || !(skip <= 1.0)) return -1;
+  long long s = static_cast<long long>(std::floor(static_cast<double>(total_steps) * skip + 1e-9));
+  if (s < 1) s = 1;
+  if (s > total_steps) s = total_steps;
+  return static_cast<int32_t>(s);
+}
+
+int32_t sparsed_schedule_mode(int32_t step_1based, int32_t total_steps, double skip) {
+  const int32_t s = sparsed_switch_step(total_steps, skip);
+  if (s < 0 || step_1based < 1 || step_1based > total_steps) return -1;
+  if (step_1based < s) return SPARSED_MODE_FULL;
+  if (step_1based == s) return SPARSED_MODE_FULL_AND_SELECT;
+  return SPARSED_MODE_SPARSE;
+}
+
+sparsed_status sparsed_kept_per_row(const sparsed_select_params* params, int32_t seq_len, int32_t* k_pre,
+                                    int32_t* k_gen) {
+  if (params == nullptr || k_pre == nullptr || k_gen == nullptr || seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+  if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  int pb = 0, a = 0, b = 0;
+  sparsed_status st = kept_counts(params, seq_len / params->block_size, &pb, &a, &b);
+  if (st != SPARSED_OK) return st;
+  *k_pre = a;
+  *k_gen = b;
+  return SPARSED_OK;
+}
+
+sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape* shape, const sparsed_select_params* params,
+                                       size_t* out_bytes) {
+  if (out_bytes == nullptr) return SPARSED_ERR_INVALID_ARG;
+  switch (op) {
+    case SPARSED_OP_ATTN_FULL:
+    case SPARSED_OP_ATTN_SPARSE:
+    case SPARSED_OP_SELECT_FROM_SCORES:
+    case SPARSED_OP_PATTERN_VALIDATE:
+      *out_bytes = SPARSED_STATUS_BYTES;
+      return SPARSED_OK;
+    case SPARSED_OP_SELECT_PATTERN: {
+      if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
+      if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+      if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+      if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+      const size_t nb = static_cast<size_t>(shape->seq_len / params->block_size);
+      const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
+      *out_bytes = SPARSED_STATUS_BYTES + round_up(bh * nb * nb * 4, 256) +
+                   round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
+      return SPARSED_OK;
+    }
+    default:
+      return SPARSED_ERR_INVALID_ARG;
+  }
+}
+
+sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  cudaError_t e = cudaMemsetAsync(ws, 0, SPARSED_STATUS_BYTES, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
+}
+
+sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
+                                 float* lse_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Resolved rs;
+  sparsed_status st = check_shape(shape, true, &rs);
+  if (st != SPARSED_OK) return st;
+  if (q == nullptr || k == nullptr || v == nullptr || o == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SPARSED_ERR_ALIGNMENT;
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_arch()) != SPARSED_OK) return st;
+  CUtensorMap tq, tk, tv;
+  if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 128)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 128)) != SPARSED_OK) return st;
+  AttnParams p;
+  p.o = o;
+  p.o_stride_b = rs.o[0];
+  p.o_stride_h = rs.o[1];
+  p.o_stride_t = rs.o[2];
+  p.lse = lse_or_null;
+  p.seq_len = shape->seq_len;
+  p.heads_q = shape->heads_q;
+  p.group = shape->heads_q / shape->heads_kv;
+  p.num_q_tiles = (shape->seq_len + 127) / 128;
+  p.scale_log2 = rs.scale_log2;
+  p.row_ptr = nullptr;
+  p.col_idx = nullptr;
+  p.status = static_cast<DeviceStatus*>(ws);
+  cudaError_t e = launch_attn_dense(tq, tk, tv, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
+}
+
+sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pattern* pattern, const void* q,
+                                   const void* k, const void* v, void* o, void* ws, size_t ws_bytes,
+                                   void* cuda_stream) {
+  Resolved rs;
+  sparsed_status st = check_shape(shape, true, &rs);
+  if (st != SPARSED_OK) return st;
+  if (q == nullptr || k == nullptr || v == nullptr || o == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SPARSED_ERR_ALIGNMENT;
+  if (pattern == nullptr || pattern->row_ptr == nullptr || pattern->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if (pattern->block_size != 64 && pattern->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (pattern->batch != shape->batch || pattern->heads_q != shape->heads_q || pattern->num_blocks < 1 ||
+      static_cast<int64_t>(pattern->num_blocks) * pattern->block_size != shape->seq_len)
+    return SPARSED_ERR_PATTERN;
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_arch()) != SPARSED_OK) return st;
+  const int bs = pattern->block_size;
+  CUtensorMap tq, tk, tv;
+  if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, bs)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, bs)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, bs)) != SPARSED_OK) return st;
+  AttnParams p;
+  p.o = o;
+  p.o_stride_b = rs.o[0];
+  p.o_stride_h = rs.o[1];
+  p.o_stride_t = rs.o[2];
+  p.lse = nullptr;
+  p.seq_len = shape->seq_len;
+  p.heads_q = shape->heads_q;
+  p.group = shape->heads_q / shape->heads_kv;
+  p.num_q_tiles = pattern->num_blocks;
+  p.scale_log2 = rs.scale_log2;
+  p.row_ptr = pattern->row_ptr;
+  p.col_idx = pattern->col_idx;
+  p.status = static_cast<DeviceStatus*>(ws);
+  cudaError_t e = launch_attn_sparse(tq, tk, tv, p, shape->batch, bs, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
+}
+
+sparsed_status sparsed_select_from_scores(const sparsed_select_params* params, const float* scores, int32_t batch,
+                                          int32_t heads_q, int32_t num_blocks, sparsed_pattern* out, void* ws,
+                                          size_t ws_bytes, void* cuda_stream) {
+  if (scores == nullptr || batch < 1 || heads_q < 1 || num_blocks < 1) return SPARSED_ERR_INVALID_ARG;
+  int pb = 0, k_pre = 0, k_gen = 0;
+  sparsed_status st = kept_counts(params, num_blocks, &pb, &k_pre, &k_gen);
+  if (st != SPARSED_OK) return st;
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  return run_topk(scores, batch, heads_q, num_blocks, params->block_size, pb, k_pre, k_gen, out,
+                  static_cast<cudaStream_t>(cuda_stream));
+}
+
+sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_select_params* params, const void* q,
+                                      const void* k, const float* lse_or_null, sparsed_pattern* out,
+                                      float* scores_out_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Resolved rs;
+  sparsed_status st = check_shape(shape, false, &rs);
+  if (st != SPARSED_OK) return st;
+  if (params == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  const int nb = shape->seq_len / params->block_size;
+  int pb = 0, k_pre = 0, k_gen = 0;
+  if ((st = kept_counts(params, nb, &pb, &k_pre, &k_gen)) != SPARSED_OK) return st;
+  if (q == nullptr || k == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return SPARSED_ERR_ALIGNMENT;
+  if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  size_t need = 0;
+  if ((st = sparsed_workspace_bytes(SPARSED_OP_SELECT_PATTERN, shape, params, &need)) != SPARSED_OK) return st;
+  const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
+  const size_t score_bytes = round_up(bh * nb * nb * 4, 256);
+  const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
+  size_t required = SPARSED_STATUS_BYTES + (scores_out_or_null ? 0 : score_bytes) + (lse_or_null ? 0 : lse_bytes);
+  if (ws == nullptr || ws_bytes < required) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_arch()) != SPARSED_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  float* scores = scores_out_or_null;
+  size_t off = SPARSED_STATUS_BYTES;
+  if (scores == nullptr) {
+    scores = reinterpret_cast<float*>(base + off);
+    off += score_bytes;
+  }
+  CUtensorMap tq, tk;
+  if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 128)) != SPARSED_OK) return st;
+  ScoreParams sp;
+  sp.scores = scores;
+  sp.lse = lse_or_null;
+  sp.seq_len = shape->seq_len;
+  sp.heads_q = shape->heads_q;
+  sp.group = shape->heads_q / shape->heads_kv;
+  sp.block_size = params->block_size;
+  sp.scale_log2 = rs.scale_log2;
+  sp.status = static_cast<DeviceStatus*>(ws);
+  if (lse_or_null == nullptr) {
+    float* lse_buf = reinterpret_cast<float*>(base + off);
+    cudaError_t e = launch_row_stats(tq, tk, sp, lse_buf, shape->batch, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    sp.lse = lse_buf;
+  }
+  cudaError_t e = launch_pooled_scores(tq, tk, sp, shape->batch, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return run_topk(scores, shape->batch, shape->heads_q, nb, params->block_size, pb, k_pre, k_gen, out, stream);
+}
+
+sparsed_status sparsed_pattern_validate(const sparsed_pattern* pattern, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (pattern == nullptr || pattern->row_ptr == nullptr || pattern->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if (pattern->batch < 1 || pattern->heads_q < 1 || pattern->num_blocks < 1) return SPARSED_ERR_PATTERN;
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  const int64_t rows = static_cast<int64_t>(pattern->batch) * pattern->heads_q * pattern->num_blocks;
+  if (rows >= INT32_MAX) return SPARSED_ERR_UNSUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int* flag = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + 16);
+  cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(int), stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_pattern_validate(pattern->row_ptr, pattern->col_idx, static_cast<int>(rows), pattern->num_blocks,
+                              pattern->col_capacity, flag, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  int host_flag = 0;
+  e = cudaMemcpyAsync(&host_flag, flag, sizeof(int), cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return host_flag == 0 ? SPARSED_OK : SPARSED_ERR_PATTERN;
+}
+
+sparsed_status sparsed_last_device_status(void* ws, void* cuda_stream, int32_t* code, int32_t* where) {
+  if (ws == nullptr) return SPARSED_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int32_t host[2] = {0, 0};
+  cudaError_t e = cudaMemcpyAsync(host, ws, sizeof(host), cudaMemcpyDeviceToHost, stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (code != nullptr) *code = host[0];
+  if (where != nullptr) *where = host[1];
+  return host[0] == 0 ? SPARSED_OK : SPARSED_ERR_DEVICE_TIMEOUT;
+}
+
+}  // extern "C"

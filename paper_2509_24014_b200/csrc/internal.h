@@ -1,0 +1,61 @@
+// Internal host-side interfaces between the C ABI layer and the kernel launchers.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sm100_primitives.cuh"
+
+namespace sparsed {
+
+// Parameters shared by the dense and the block-sparse attention kernels.
+struct AttnParams {
+  void* o;                 // bf16 [B,Hq,L,D]
+  int64_t o_stride_b, o_stride_h, o_stride_t;
+  float* lse;              // fp32 [B,Hq,L] or null
+  int seq_len;
+  int heads_q;
+  int group;               // heads_q / heads_kv
+  int num_q_tiles;         // query tiles per (batch, head)
+  float scale_log2;        // softmax scale * log2(e)
+  const int32_t* row_ptr;  // sparse only
+  const int32_t* col_idx;  // sparse only
+  DeviceStatus* status;
+};
+
+// Parameters of the pooled-scoring kernel.
+struct ScoreParams {
+  float* scores;           // fp32 [B,Hq,nb,nb]
+  const float* lse;        // fp32 [B,Hq,L], natural log
+  int seq_len;
+  int heads_q;
+  int group;
+  int block_size;          // 64 or 128
+  float scale_log2;
+  DeviceStatus* status;
+};
+
+struct TopkParams {
+  const float* scores;     // fp32 [rows, nb]
+  int32_t* row_ptr;
+  int32_t* col_idx;
+  int rows;                // B * Hq * nb
+  int nb;
+  int pb;                  // prefill blocks
+  int k_pre, k_gen;
+};
+
+cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                              const AttnParams& p, int batch, cudaStream_t stream);
+cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                               const AttnParams& p, int batch, int block_size, cudaStream_t stream);
+cudaError_t launch_row_stats(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, float* lse_out,
+                             int batch, cudaStream_t stream);
+cudaError_t launch_pooled_scores(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int batch,
+                                 cudaStream_t stream);
+cudaError_t launch_topk_csr(const TopkParams& p, cudaStream_t stream);
+cudaError_t launch_pattern_validate(const int32_t* row_ptr, const int32_t* col_idx, int rows, int nb,
+                                    int64_t capacity, int* bad_flag, cudaStream_t stream);
+
+}  // namespace sparsed
