@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the SparseD attention hot path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic batch of the 64k workload:
+schedule helper -> dense attention (+LSE) -> pattern selection (pooled scoring, top-k, CSR)
+-> block-sparse attention on the selected pattern. The headline value is the block-sparse
+attention throughput in TFLOP/s counted on kept-block FLOPs (4 * bs^2 * D * nnz), with its
+fraction of the measured bf16 peak and the wall-time speedup over the library's own dense
+kernel reported beside it.
+
+    python bench.py --gpus 1 --steps 5 --warmup 3            # this library
+    python bench.py --impl reference --steps 2 --warmup 1     # the CPU oracle on host cores
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica of the workload
+(the path has no exchange step); value = work of all ranks / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_24014_b200 import synthetic as syn  # noqa: E402
+
+METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at 64k"
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; keyed by (kernel, workload). None where no capture exists.
+NCU_DRAM_TRAFFIC = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def sparse_flops(cfg, nnz):
+    return 4.0 * cfg.block_size * cfg.block_size * cfg.head_dim * nnz
+
+
+def dense_flops(cfg):
+    return 4.0 * cfg.seq_len * cfg.seq_len * cfg.head_dim * cfg.heads_q * cfg.batch
+
+
+# ------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sparse_sample(cfg, q, k, v, rp, ci, n_row_blocks, seed=0):
+    """Times the fp64 oracle's masked attention on a seeded sample of (head, query block) rows.
+    Returns (kept-block TFLOP/s, seconds, rows, threads)."""
+    from oracle import sparsed_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    rng = np.random.default_rng(seed)
+    nb = cfg.num_blocks
+    group = cfg.heads_q // cfg.heads_kv
+    heads = rng.integers(0, cfg.heads_q, n_row_blocks)
+    blocks = rng.integers(0, nb, n_row_blocks)
+    cache = {}
+    flops = 0.0
+    t_total = 0.0
+    for h, ib in zip(heads, blocks):
+        hk = int(h) // group
+        if ("k", hk) not in cache:
+            cache.clear()
+            cache[("k", hk)] = (k[0, hk].to(torch.float64).numpy(), v[0, hk].to(torch.float64).numpy())
+        kh, vh = cache[("k", hk)]
+        qh = q[0, int(h)].to(torch.float64).numpy()
+        r = int(h) * nb + int(ib)
+        kept = ci[rp[r]:rp[r + 1]]
+        t0 = time.perf_counter()
+        orc.head_sparse_rows(qh, kh, vh, int(ib), kept, cfg.block_size)
+        t_total += time.perf_counter() - t0
+        flops += 4.0 * cfg.block_size * cfg.block_size * cfg.head_dim * len(kept)
+    return flops / t_total / 1e12, t_total, n_row_blocks, threads
+
+
+def run_reference(args, cfg):
+    """The oracle as it stands, timed on the host cores, on bounded samples of the workload."""
+    from oracle import sparsed_oracle as orc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    small = cfg.with_(heads_q=2, heads_kv=2 if cfg.heads_kv == cfg.heads_q else 1)
+    q, k, v = syn.make_qkv(small, "cpu")
+    nb = cfg.num_blocks
+    pb = cfg.prefill_len // cfg.block_size
+    k_pre, k_gen = orc.kept_per_region(pb, cfg.keep_ratio), orc.kept_per_region(nb - pb, cfg.keep_ratio)
+    kh, vh = k[0, 0].to(torch.float64).numpy(), v[0, 0].to(torch.float64).numpy()
+    qh = q[0, 0].to(torch.float64).numpy()
+    rows_per_step = args.ref_rows
+    rng = np.random.default_rng(0)
+
+    def one_step():
+        flops = 0.0
+        for _ in range(rows_per_step):
+            ib = int(rng.integers(0, nb))
+            # select this row block's pattern with the oracle itself, then attend
+            kept = orc.select_row(orc.head_pooled_row(qh, kh, ib, cfg.block_size), pb, cfg.keep_ratio)
+            t0 = time.perf_counter()
+            orc.head_sparse_rows(qh, kh, vh, ib, kept, cfg.block_size)
+            one_step.sparse_s += time.perf_counter() - t0
+            flops += 4.0 * cfg.block_size ** 2 * cfg.head_dim * len(kept)
+        return flops
+
+    one_step.sparse_s = 0.0
+    for _ in range(args.warmup):
+        one_step()
+    one_step.sparse_s = 0.0
+    t0 = time.perf_counter()
+    flops = 0.0
+    for _ in range(args.steps):
+        flops += one_step()
+    wall = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    value = flops / one_step.sparse_s / 1e12
+    sample = (f"{rows_per_step} seeded (head, query block) rows of {cfg.heads_q * nb} per step; each row: oracle "
+              f"scoring+selection (untimed) then oracle masked attention (timed), k={k_pre}+{k_gen} of {nb} blocks")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": workload_name(cfg), "timing": "host perf_counter"},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_name(cfg):
+    return (f"{cfg.name}: B{cfg.batch} Hq{cfg.heads_q}/Hkv{cfg.heads_kv} L{cfg.seq_len} D{cfg.head_dim} bf16, "
+            f"block {cfg.block_size}, keep {cfg.keep_ratio}, prefill {cfg.prefill_len}")
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def run_ours(args, cfg):
+    import paper_2509_24014_b200 as sd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    sd.load_library()
+    peaks = load_peaks()
+
+    cfg_r = cfg.with_(seed=cfg.seed + 1000 * rank)
+    q, k, v = syn.make_qkv(cfg_r, dev)
+    B, Hq, L, D = q.shape
+    nb = cfg.num_blocks
+    o_full = torch.empty_like(q)
+    o_sparse = torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+    params = sd.make_params(cfg.block_size, cfg.keep_ratio, cfg.prefill_len)
+    k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
+    pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+    shape_qkvo = sd.make_shape(q, k, v, o_full)
+    shape_qk = sd.make_shape(q, k)
+    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_PATTERN, shape_qk, params), dev)
+    total_steps, skip = max(cfg.total_steps, 2), (cfg.skip if cfg.total_steps > 1 else 0.5)
+    s_switch = sd.sparsed_switch_step(total_steps, skip)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(events=None):
+        """All rows of the hot path once. Returns nothing; `events` collects 5 stream markers."""
+        marks = []
+        def mark():
+            if events is not None:
+                e = ev(); e.record(); marks.append(e)
+        mark()
+        assert sd.sparsed_schedule_mode(s_switch, total_steps, skip) == sd.MODE_FULL_AND_SELECT
+        sd.sparsed_attn_full(q, k, v, o_full, lse, ws, shape=shape_qkvo)
+        mark()
+        sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse, shape=shape_qk)
+        mark()
+        assert sd.sparsed_schedule_mode(s_switch + 1, total_steps, skip) == sd.MODE_SPARSE
+        sd.sparsed_attn_sparse(q, k, v, o_sparse, pat, ws, shape=shape_qkvo)
+        mark()
+        if events is not None:
+            events.append(marks)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    events = []
+    t_begin, t_end = ev(), ev()
+    t_begin.record()
+    for _ in range(args.steps):
+        step(events)
+    t_end.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    code, where = sd.sparsed_last_device_status(ws)
+    if code != 0:
+        raise RuntimeError(f"device status {code} at {where}")
+
+    full_ms = [m[0].elapsed_time(m[1]) for m in events]
+    select_ms = [m[1].elapsed_time(m[2]) for m in events]
+    sparse_ms = [m[2].elapsed_time(m[3]) for m in events]
+    sparse_total = sum(sparse_ms)
+    nnz = int(pat.nnz)
+
+    # max over ranks of the timed quantities
+    if dist is not None:
+        t = torch.tensor([total_ms, sparse_total, sum(full_ms), sum(select_ms)], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, sparse_total, full_total, select_total = t.tolist()
+    else:
+        full_total, select_total = sum(full_ms), sum(select_ms)
+
+    n = args.steps
+    value = world * n * sparse_flops(cfg, nnz) / (sparse_total * 1e-3) / 1e12
+    dense_tflops = world * n * dense_flops(cfg) / (full_total * 1e-3) / 1e12
+    per_gpu_sparse = value / world
+    per_gpu_dense = dense_tflops / world
+
+    # ---- end to end through the public API with host buffers (rank-local, then max) -------
+    e2e_steps = max(1, min(args.steps, 3))
+    hq, hk, hv = (t.to("cpu").pin_memory() for t in (q, k, v))
+    ho = torch.empty(o_sparse.shape, dtype=o_sparse.dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+    d2h = ho.numel() * ho.element_size()
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    def e2e_once():
+        q.copy_(hq, non_blocking=True); k.copy_(hk, non_blocking=True); v.copy_(hv, non_blocking=True)
+        sd.sparsed_attn_sparse(q, k, v, o_sparse, pat, ws, shape=shape_qkvo)
+        ho.copy_(o_sparse, non_blocking=True)
+    e2e_once()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_once()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = t.item()
+    e2e_value = world * e2e_steps * sparse_flops(cfg, nnz) / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak = peaks["bf16_tflops"]
+    tag = "of measured" if peaks["source"] == "measured" else "of fallback"
+
+    def tensor_roofline(name, flops_per_launch, ms_list, launches_per_step=1):
+        ms = sum(ms_list) / (len(ms_list) * launches_per_step)
+        ach = flops_per_launch / (ms * 1e-3) / 1e12
+        return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                "frac": ach / peak, "peak_source": f"bf16 burst, {tag}",
+                "frac_of_sustained": ach / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
+                "avg_launch_ms": ms, "traffic": NCU_DRAM_TRAFFIC.get((name, cfg.name))}
+
+    roof_dense = tensor_roofline("attn_kernel<dense>", dense_flops(cfg), full_ms)
+    roof_sparse = tensor_roofline("attn_kernel<sparse>", sparse_flops(cfg, nnz), sparse_ms)
+    # selection = pooled-scoring kernel (a dense QK^T contraction, 2*L^2*D per head) + top-k/CSR kernel
+    roof_select = tensor_roofline("score_kernel+topk_csr_kernel", dense_flops(cfg) / 2, select_ms)
+    dominant = max((roof_dense, roof_select, roof_sparse), key=lambda r: r["avg_launch_ms"])
+
+    # ---- CPU oracle beside it (bounded sample of the same workload) ----------------------
+    cpu = None
+    if not args.no_cpu_baseline:
+        rp_h = row_ptr.cpu().numpy()
+        ci_h = col_idx.cpu().numpy()
+        n_rows = args.cpu_rows
+        val, secs, rows, threads = oracle_sparse_sample(cfg, hq, hk, hv, rp_h, ci_h, n_rows)
+        cpu = {"value": val, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+               "sample": f"oracle masked attention (fp64 numpy) on {rows} seeded (head, query block) rows of "
+                         f"{Hq * nb}, GPU-selected pattern, {secs:.1f} s; kept-block FLOPs / time",
+               "seconds": secs, "host_cpus": os.cpu_count()}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": n, "warmup": args.warmup,
+        "ms_per_step": total_ms / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "step": "attn_full+lse -> select_pattern -> attn_sparse",
+                   "kept_per_row": [k_pre, k_gen], "nnz": nnz, "density": nnz / (B * Hq * nb * nb),
+                   "l2": "inputs larger than L2 (Q,K,V,O = %.2f GB per pass)" % (4 * q.numel() * 2 / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "pct_bf16_peak": 100.0 * per_gpu_sparse / peak,
+        "pct_bf16_peak_sustained": 100.0 * per_gpu_sparse / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
+        "pct_bf16_nominal_2250": 100.0 * per_gpu_sparse / 2250.0,
+        "dense_tflops": dense_tflops,
+        "speedup_vs_dense": full_total / sparse_total, "ideal_speedup": nb / (k_pre + k_gen),
+        "phase_ms": {"attn_full": full_total / n, "select_pattern": select_total / n, "attn_sparse": sparse_total / n},
+        "roofline": dominant, "roofline_by_kernel": [roof_dense, roof_select, roof_sparse],
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "what": "pinned host Q,K,V -> device, sparsed_attn_sparse, O -> pinned host", "steps": e2e_steps,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": 4 * n, "launches_per_step": {"attn_kernel<dense>": 1, "score_kernel": 1,
+                                                     "topk_csr_kernel": 1, "attn_kernel<sparse>": 1},
+        "clocks": clocks, "peaks": peaks,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c4", choices=sorted(syn.CONFIGS))
+    ap.add_argument("--cpu-rows", type=int, default=160, help="row blocks the CPU oracle is timed on")
+    ap.add_argument("--ref-rows", type=int, default=4, help="row blocks per step of the reference arm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = syn.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
