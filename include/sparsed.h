@@ -167,6 +167,35 @@ sparsed_status sparsed_pattern_validate(const sparsed_pattern *pattern, void *ws
  * `where` identifies the wait. Returns SPARSED_ERR_DEVICE_TIMEOUT if code != 0. */
 sparsed_status sparsed_last_device_status(void *ws, void *cuda_stream, int32_t *code, int32_t *where);
 
+/*
+ * sparsed_select_pattern for callers that cannot give it a workspace because they cannot
+ * allocate device memory at this point: for example a serving process whose own pool took
+ * all of the GPU's memory at start-up (a later cudaMalloc would fail), or a request path
+ * on which allocation is banned because cudaMalloc and cudaFree stall the whole device.
+ * (The paper has no counterpart; this is a deployment convenience.)
+ *
+ * Same inputs, outputs, rules and errors as sparsed_select_pattern with scores_out = NULL,
+ * but the scratch (status block, pooled scores, and the LSE rows if lse_or_null is NULL)
+ * is a fixed array of SPARSED_STATIC_SCRATCH_BYTES inside the library's device image, which
+ * every GPU that loads the library holds until the process exits. The call allocates and
+ * frees nothing, on the device or through any library.
+ *  - Limit: sparsed_workspace_bytes(SPARSED_OP_SELECT_PATTERN, ...) minus the LSE part when
+ *    an LSE is passed must not exceed SPARSED_STATIC_SCRATCH_BYTES, else the call returns
+ *    SPARSED_ERR_WORKSPACE and launches nothing (use sparsed_select_pattern instead).
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call before any stream capture begins.
+ *  - All calls on a device share the one array: calls that can overlap on the GPU (different
+ *    streams, different threads) race on it. Serialise them. The array keeps the previous
+ *    call's contents; the call itself re-zeroes the part that has to start at zero.
+ *  - Device-side wait timeouts of this variant are recorded in the internal array, which
+ *    sparsed_last_device_status cannot read; check the pattern with sparsed_pattern_validate
+ *    if in doubt.
+ */
+#define SPARSED_STATIC_SCRATCH_BYTES (8u << 20)
+sparsed_status sparsed_select_pattern_static(const sparsed_shape *shape, const sparsed_select_params *params,
+                                             const void *q, const void *k, const float *lse_or_null,
+                                             sparsed_pattern *out, void *cuda_stream);
+
 const char *sparsed_status_string(sparsed_status status);
 int32_t sparsed_last_cuda_error(void);
 

@@ -4,6 +4,6 @@ from .binding import (  # noqa: F401
     OP_SELECT_FROM_SCORES, OP_SELECT_PATTERN, Pattern, SelectParams, Shape, SparsedError, load_library,
     make_params, make_shape, new_pattern, new_workspace, pattern_from_csr, sparsed_attn_full, sparsed_attn_sparse,
     sparsed_kept_per_row, sparsed_last_device_status, sparsed_pattern_validate, sparsed_schedule_mode,
-    sparsed_select_from_scores, sparsed_select_pattern, sparsed_switch_step, sparsed_workspace_bytes,
+    sparsed_select_from_scores, sparsed_select_pattern, sparsed_select_pattern_static, sparsed_switch_step, sparsed_workspace_bytes,
     sparsed_workspace_init,
 )

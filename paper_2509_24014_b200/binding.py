@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_attn_full", "sparsed_select_pattern", "sparsed_select_from_scores", "sparsed_attn_sparse",
     "sparsed_schedule_mode", "sparsed_switch_step", "sparsed_kept_per_row", "sparsed_workspace_bytes",
     "sparsed_workspace_init", "sparsed_pattern_validate", "sparsed_last_device_status",
-    "sparsed_status_string", "sparsed_last_cuda_error",
+    "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
 )
 
 
@@ -73,6 +73,7 @@ def load_library() -> ctypes.CDLL:
     P = ctypes.POINTER
     lib.sparsed_attn_full.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_pattern.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp, vp, sz, vp]
+    lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
     lib.sparsed_select_from_scores.argtypes = [P(SelectParams), vp, i32, i32, i32, P(Pattern), vp, sz, vp]
     lib.sparsed_attn_sparse.argtypes = [P(Shape), P(Pattern), vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_schedule_mode.argtypes = [i32, i32, f64]
@@ -199,6 +200,21 @@ def sparsed_select_pattern(q, k, params: SelectParams, pattern: Pattern, ws: tor
         lse.data_ptr() if lse is not None else None, ctypes.byref(pattern),
         scores_out.data_ptr() if scores_out is not None else None, ws.data_ptr(), ws.numel(), _stream(q)),
         "sparsed_select_pattern")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def sparsed_select_pattern_static(q, k, params: SelectParams, pattern: Pattern, lse: Optional[torch.Tensor] = None,
+                                  softmax_scale: float = 0.0, shape: Optional[Shape] = None) -> None:
+    """Pattern selection for callers that may not allocate device memory: the scratch is a fixed
+    array inside the library (STATIC_SCRATCH_BYTES), shared by every call on the device, so
+    calls must not overlap on the GPU. Requests that do not fit raise SparsedError (status 4)."""
+    shape = shape or make_shape(q, k, None, None, softmax_scale)
+    _check(load_library().sparsed_select_pattern_static(
+        ctypes.byref(shape), ctypes.byref(params), q.data_ptr(), k.data_ptr(),
+        lse.data_ptr() if lse is not None else None, ctypes.byref(pattern), _stream(q)),
+        "sparsed_select_pattern_static")
 
 
 def sparsed_select_from_scores(scores: torch.Tensor, params: SelectParams, pattern: Pattern,

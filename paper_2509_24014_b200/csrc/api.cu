@@ -425,3 +425,62 @@ sparsed_status sparsed_last_device_status(void* ws, void* cuda_stream, int32_t* 
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Selection without a caller workspace: the scratch lives in this library's device image.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticScratchBytes = SPARSED_STATIC_SCRATCH_BYTES;
+
+// Scratch for sparsed_select_pattern_static: status block, pooled scores A', and the LSE
+// rows when the caller has none. One copy per GPU that loads the library, held until exit.
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticScratchBytes];
+
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[64] = {};
+
+// In host code `g_select_scratch` is only a handle for the runtime, not a device address:
+// the address a kernel may use is looked up once per device with that device current.
+sparsed_status static_scratch_address(void** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return SPARSED_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (g_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_select_scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (ptr == nullptr) return cuda_fail(cudaErrorInvalidSymbol);
+    g_scratch_addr[dev] = ptr;
+  }
+  *out = g_scratch_addr[dev];
+  return SPARSED_OK;
+}
+
+}  // namespace
+
+extern "C" sparsed_status sparsed_select_pattern_static(const sparsed_shape* shape,
+                                                        const sparsed_select_params* params, const void* q,
+                                                        const void* k, const float* lse_or_null,
+                                                        sparsed_pattern* out, void* cuda_stream) {
+  if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
+  // Size check first, on the host, so that an oversized request never reaches the device.
+  size_t full = 0;
+  sparsed_status st = sparsed_workspace_bytes(SPARSED_OP_SELECT_PATTERN, shape, params, &full);
+  if (st != SPARSED_OK) return st;
+  const size_t bh = static_cast<size_t>(shape->batch) * static_cast<size_t>(shape->heads_q);
+  const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
+  const size_t needed = full - (lse_or_null != nullptr ? lse_bytes : 0);
+  if (needed > kStaticScratchBytes) return SPARSED_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  if ((st = static_scratch_address(&scratch)) != SPARSED_OK) return st;
+  // The array keeps whatever the previous call left: the status block must start at zero;
+  // scores and LSE rows are fully rewritten by the kernels before anything reads them.
+  cudaError_t e = cudaMemsetAsync(scratch, 0, SPARSED_STATUS_BYTES, static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return cuda_fail(e);
+  return sparsed_select_pattern(shape, params, q, k, lse_or_null, out, nullptr, scratch, kStaticScratchBytes,
+                                cuda_stream);
+}
+
