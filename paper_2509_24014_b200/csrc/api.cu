@@ -266,8 +266,8 @@ sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, cons
   if ((st = check_arch()) != SPARSED_OK) return st;
   CUtensorMap tq, tk, tv;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 128)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 128)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 64)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 64)) != SPARSED_OK) return st;
   AttnParams p;
   p.o = o;
   p.o_stride_b = rs.o[0];
@@ -304,8 +304,8 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   const int bs = pattern->block_size;
   CUtensorMap tq, tk, tv;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, bs)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, bs)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, bs)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 64)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 64)) != SPARSED_OK) return st;
   AttnParams p;
   p.o = o;
   p.o_stride_b = rs.o[0];

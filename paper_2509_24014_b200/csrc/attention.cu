@@ -1,53 +1,61 @@
 // Dense bidirectional attention (Eq. 1 times V) and block-sparse attention (Eq. 3 / Eq. 4
 // times V) for head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a.
 //
-// One CTA owns one query tile of one (batch, head) and streams key/value tiles through a
+// One CTA owns one query tile of one (batch, head) and streams 64-key tiles through a
 // warp-specialised pipeline:
-//   warp 4  : TMA producer  - Q once, then a K tile and a V tile per step (128B-swizzled smem)
-//   warp 5  : UMMA issuer   - S = Q K^T into tensor memory, then O += P V with P read from
-//                             tensor memory (P overwrites the first half of S's columns)
-//   warps 0-3: one thread per query row - online softmax in fp32 on the scaled base-2 logits,
-//             writes P as bf16 into tensor memory, rescales O only when the running row
-//             maximum grew by more than 2^8, and finally normalises and stores O (and LSE).
+//   warp 4  : TMA producer  - Q once, then a K tile and a V tile per step into two-stage
+//                             rings of 128B-swizzled shared memory
+//   warp 5  : UMMA issuer   - S_j = Q K_j^T into one of two tensor-memory buffers, then
+//                             O += P_j V_j with P read from tensor memory (P overwrites the
+//                             first half of S_j's columns). S_{j+1} is issued before P_j V_j,
+//                             so the tensor pipe works on the next logits while the softmax
+//                             warps are busy with the current ones.
+//   warps 0-3: one thread per query row - online softmax in fp32 on base-2 logits. The tile
+//             is exponentiated once against the running maximum; only if some row's maximum
+//             grew by more than 2^8 is the tile redone with the new maximum and O rescaled
+//             (after the previous P V has drained). Finally O is normalised and stored.
 // The dense kernel walks all key tiles; the sparse kernel walks the CSR list of its query
-// block. Two CTAs fit on one SM (96 KB of shared memory, 256 tensor-memory columns each), so
-// one CTA's softmax overlaps the other's tensor-core work.
+// block (a 128-key block is two consecutive tiles). Two CTAs fit on one SM (96 KB of shared
+// memory and 256 tensor-memory columns each).
 #include "internal.h"
 
 namespace sparsed {
 namespace {
 
 constexpr int kHeadDim = 128;
-constexpr int kTileM = 128;        // UMMA M; rows of tensor memory
+constexpr int kTileM = 128;   // UMMA M; rows of tensor memory
+constexpr int kTileN = 64;    // keys per pipeline step
+constexpr int kStages = 2;    // K and V ring depth
 constexpr int kSoftmaxThreads = 128;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
-constexpr int kColS = 0;           // S (fp32) and P (bf16 pairs) live here
-constexpr int kColO = 128;         // O accumulator (fp32)
+constexpr int kColS = 0;      // two S buffers of 64 fp32 columns; P (bf16 pairs) reuses the first 32
+constexpr int kColO = 128;    // O accumulator (fp32, 128 columns)
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
 
-template <int kBlockN>
 struct AttnSmem {
-  alignas(1024) __nv_bfloat16 q[2][kTileM * 64];
-  alignas(1024) __nv_bfloat16 k[2][kBlockN * 64];
-  alignas(1024) __nv_bfloat16 v[2][kBlockN * 64];
-  uint64_t q_full, k_full, k_empty, v_full, v_empty, s_full, p_full, o_full;
+  alignas(1024) __nv_bfloat16 q[2][kTileM * 64];           // two 64-wide halves of head_dim
+  alignas(1024) __nv_bfloat16 k[kStages][2][kTileN * 64];
+  alignas(1024) __nv_bfloat16 v[kStages][2][kTileN * 64];
+  uint64_t q_full, k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t s_full[2], p_full[2], o_full;
   uint32_t tmem_base;
   int abort_flag;
 };
 
-// kBlockN : keys per tile (64 or 128).  kRowsQ : valid query rows per tile (64 or 128).
-template <int kBlockN, int kRowsQ, bool kSparse>
+// kSparse : walk the CSR list instead of all keys.  kBlock : keys per pattern block (sparse).
+// kRowsQ  : valid query rows per tile (64 or 128; the UMMA tile is always 128 rows).
+template <bool kSparse, int kBlock, int kRowsQ>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
-  using Smem = AttnSmem<kBlockN>;
-  Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  AttnSmem& sm = *reinterpret_cast<AttnSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
   const int lane = tid & 31;
+  constexpr int kTilesPerBlock = kBlock / kTileN;
 
   // ---- work item -----------------------------------------------------------------------
   const int q_tile = blockIdx.x % p.num_q_tiles;
@@ -57,24 +65,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const int kv_head = head / p.group;
   const int q_row0 = q_tile * kRowsQ;
 
-  int tile_begin = 0, num_tiles;
+  int list_begin = 0, num_tiles;
   if constexpr (kSparse) {
     const int r = bh * p.num_q_tiles + q_tile;
-    tile_begin = __ldg(p.row_ptr + r);
-    num_tiles = __ldg(p.row_ptr + r + 1) - tile_begin;
+    list_begin = __ldg(p.row_ptr + r);
+    num_tiles = (__ldg(p.row_ptr + r + 1) - list_begin) * kTilesPerBlock;
   } else {
-    num_tiles = (p.seq_len + kBlockN - 1) / kBlockN;
+    num_tiles = (p.seq_len + kTileN - 1) / kTileN;
   }
 
   // ---- set-up --------------------------------------------------------------------------
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    mbar_init(&sm.k_full, 1);
-    mbar_init(&sm.k_empty, 1);
-    mbar_init(&sm.v_full, 1);
-    mbar_init(&sm.v_empty, 1);
-    mbar_init(&sm.s_full, 1);
-    mbar_init(&sm.p_full, kSoftmaxThreads);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.k_full[s], 1);
+      mbar_init(&sm.k_empty[s], 1);
+      mbar_init(&sm.v_full[s], 1);
+      mbar_init(&sm.v_empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.s_full[s], 1);
+      mbar_init(&sm.p_full[s], kSoftmaxThreads);
+    }
     mbar_init(&sm.o_full, 1);
     sm.abort_flag = 0;
     mbar_fence_init();
@@ -98,7 +110,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
-  const uint32_t tS = tmem + kColS;
   const uint32_t tO = tmem + kColO;
 
   if (warp == 4) {
@@ -110,53 +121,71 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       mbar_expect_tx(&sm.q_full, kRowsQ * kHeadDim * 2);
       tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
       tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
-      for (int it = 0; it < num_tiles; ++it) {
-        int kv_tile;
-        if constexpr (kSparse) kv_tile = __ldg(p.col_idx + tile_begin + it);
-        else kv_tile = it;
-        const int kv_row0 = kv_tile * kBlockN;
-        if (it > 0 && !mbar_wait(&sm.k_empty, (it - 1) & 1, &sm.abort_flag, p.status, 10)) break;
-        mbar_expect_tx(&sm.k_full, kBlockN * kHeadDim * 2);
-        tma_load_4d(sm.k[0], &tm_k, &sm.k_full, 0, kv_row0, kv_head, batch);
-        tma_load_4d(sm.k[1], &tm_k, &sm.k_full, 64, kv_row0, kv_head, batch);
-        if (it > 0 && !mbar_wait(&sm.v_empty, (it - 1) & 1, &sm.abort_flag, p.status, 11)) break;
-        mbar_expect_tx(&sm.v_full, kBlockN * kHeadDim * 2);
-        tma_load_4d(sm.v[0], &tm_v, &sm.v_full, 0, kv_row0, kv_head, batch);
-        tma_load_4d(sm.v[1], &tm_v, &sm.v_full, 64, kv_row0, kv_head, batch);
+      int block_id = 0;
+      for (int t = 0; t < num_tiles; ++t) {
+        int kv_row0;
+        if constexpr (kSparse) {
+          if (t % kTilesPerBlock == 0) block_id = __ldg(p.col_idx + list_begin + t / kTilesPerBlock);
+          kv_row0 = block_id * kBlock + (t % kTilesPerBlock) * kTileN;
+        } else {
+          kv_row0 = t * kTileN;
+        }
+        const int s = t % kStages;
+        const int use = t / kStages;
+        if (use > 0 && !mbar_wait(&sm.k_empty[s], (use - 1) & 1, &sm.abort_flag, p.status, 10)) break;
+        mbar_expect_tx(&sm.k_full[s], kTileN * kHeadDim * 2);
+        tma_load_4d(sm.k[s][0], &tm_k, &sm.k_full[s], 0, kv_row0, kv_head, batch);
+        tma_load_4d(sm.k[s][1], &tm_k, &sm.k_full[s], 64, kv_row0, kv_head, batch);
+        if (use > 0 && !mbar_wait(&sm.v_empty[s], (use - 1) & 1, &sm.abort_flag, p.status, 11)) break;
+        mbar_expect_tx(&sm.v_full[s], kTileN * kHeadDim * 2);
+        tma_load_4d(sm.v[s][0], &tm_v, &sm.v_full[s], 0, kv_row0, kv_head, batch);
+        tma_load_4d(sm.v[s][1], &tm_v, &sm.v_full[s], 64, kv_row0, kv_head, batch);
       }
     }
   } else if (warp == 5) {
     // =============================== UMMA issuer ========================================
     if (lane == 0 && num_tiles > 0) {
-      constexpr uint32_t idesc_qk = umma_idesc_bf16(kTileM, kBlockN, false, false);
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(kTileM, kTileN, false, false);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(kTileM, kHeadDim, false, true);
       const uint32_t q_addr[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
-      const uint32_t k_addr[2] = {smem_u32(sm.k[0]), smem_u32(sm.k[1])};
-      const uint32_t v_addr = smem_u32(sm.v[0]);
-      bool ok = mbar_wait(&sm.q_full, 0, &sm.abort_flag, p.status, 20);
-      for (int it = 0; ok && it < num_tiles; ++it) {
-        const uint32_t ph = it & 1;
-        if (!mbar_wait(&sm.k_full, ph, &sm.abort_flag, p.status, 21)) break;
+      // S_t = Q K_t^T into S buffer t & 1
+      auto issue_qk = [&](int t) -> bool {
+        const int s = t % kStages;
+        if (!mbar_wait(&sm.k_full[s], (t / kStages) & 1, &sm.abort_flag, p.status, 21)) return false;
         tc_fence_after();
+        const uint32_t k_addr[2] = {smem_u32(sm.k[s][0]), smem_u32(sm.k[s][1])};
+        const uint32_t tS = tmem + kColS + (t & 1) * kTileN;
 #pragma unroll
         for (int kk = 0; kk < kHeadDim / 16; ++kk) {
           const uint32_t off = (kk & 3) * 32;
           umma_ss(tS, umma_smem_desc_sw128(q_addr[kk >> 2] + off, 16, 1024),
                   umma_smem_desc_sw128(k_addr[kk >> 2] + off, 16, 1024), idesc_qk, kk > 0);
         }
-        umma_commit(&sm.k_empty);
-        umma_commit(&sm.s_full);
-        if (!mbar_wait(&sm.p_full, ph, &sm.abort_flag, p.status, 22)) break;
-        if (!mbar_wait(&sm.v_full, ph, &sm.abort_flag, p.status, 23)) break;
+        umma_commit(&sm.k_empty[s]);
+        umma_commit(&sm.s_full[t & 1]);
+        return true;
+      };
+      bool ok = mbar_wait(&sm.q_full, 0, &sm.abort_flag, p.status, 20);
+      ok = ok && issue_qk(0);
+      for (int t = 0; ok && t < num_tiles; ++t) {
+        // The S buffer of tile t+1 last held P_{t-1}, whose P V was issued one iteration ago,
+        // and tcgen05 operations of one thread execute in issue order.
+        if (t + 1 < num_tiles && !issue_qk(t + 1)) break;
+        const int s = t % kStages;
+        const uint32_t ph = (t >> 1) & 1;
+        if (!mbar_wait(&sm.p_full[t & 1], ph, &sm.abort_flag, p.status, 22)) break;
+        if (!mbar_wait(&sm.v_full[s], (t / kStages) & 1, &sm.abort_flag, p.status, 23)) break;
         tc_fence_after();
+        const uint32_t v_addr = smem_u32(sm.v[s][0]);
+        const uint32_t tP = tmem + kColS + (t & 1) * kTileN;
 #pragma unroll
-        for (int kk = 0; kk < kBlockN / 16; ++kk) {
-          // V tile is [key][d]: MN-major B operand; 64-wide d halves are kBlockN*128 bytes apart
-          umma_ts(tO, tS + kk * 8, umma_smem_desc_sw128(v_addr + kk * 2048, kBlockN * 128, 1024), idesc_pv,
-                  (it > 0) || (kk > 0));
+        for (int kk = 0; kk < kTileN / 16; ++kk) {
+          // V tile is [key][d]: MN-major B operand; the two 64-wide d halves are kTileN*128 bytes apart
+          umma_ts(tO, tP + kk * 8, umma_smem_desc_sw128(v_addr + kk * 2048, kTileN * 128, 1024), idesc_pv,
+                  (t > 0) || (kk > 0));
         }
-        umma_commit(&sm.v_empty);
-        if (it == num_tiles - 1) umma_commit(&sm.o_full);
+        umma_commit(&sm.v_empty[s]);
+        if (t == num_tiles - 1) umma_commit(&sm.o_full);
       }
     }
   } else {
@@ -166,84 +195,101 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     float m_used = -INFINITY;
     float l = 0.f;
     bool ok = true;
-    for (int it = 0; it < num_tiles; ++it) {
-      if (!mbar_wait(&sm.s_full, it & 1, &sm.abort_flag, p.status, 30)) {
+    for (int t = 0; t < num_tiles; ++t) {
+      if (!mbar_wait(&sm.s_full[t & 1], (t >> 1) & 1, &sm.abort_flag, p.status, 30)) {
         ok = false;
         break;
       }
       tc_fence_after();
-      int valid_cols = kBlockN;
+      const uint32_t tS = tmem + kColS + (t & 1) * kTileN + lane_base;
+      uint32_t r0[32], r1[32];
+      tmem_ld32(tS, r0);
+      tmem_ld32(tS + 32, r1);
+      tmem_wait_ld();
       if constexpr (!kSparse) {
-        if (it == num_tiles - 1) valid_cols = p.seq_len - it * kBlockN;
-      }
-      // pass 1: row maximum of the raw logits of this tile
-      float mx = -INFINITY;
+        const int valid_cols = p.seq_len - t * kTileN;  // only the last tile can be ragged
+        if (valid_cols < kTileN) {
 #pragma unroll
-      for (int c = 0; c < kBlockN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tS + lane_base + c * 32, r);
-        tmem_wait_ld();
-        if (valid_cols >= (c + 1) * 32) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(r[j]));
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c * 32 + j < valid_cols) mx = fmaxf(mx, __uint_as_float(r[j]));
+          for (int j = 0; j < 32; ++j) {
+            if (j >= valid_cols) r0[j] = 0xff800000u;       // -inf
+            if (32 + j >= valid_cols) r1[j] = 0xff800000u;
+          }
         }
       }
-      const float m_tile = mx * scale_log2;
-      bool need = false;
-      float alpha = 1.f;
-      if (it == 0) {
-        m_used = m_tile;
-      } else {
-        need = (m_tile - m_used) > kRescaleThreshold;
-      }
-      const bool any_need = __any_sync(0xffffffffu, need);
-      if (need) {
-        alpha = fast_exp2(m_used - m_tile);
-        m_used = m_tile;
-        l *= alpha;
-      }
-      // pass 2: p = 2^(s*scale - m), row sum, bf16 P into tensor memory (over S's first columns)
-      float sum = 0.f;
+      // one pass against the running maximum: p = 2^(s*scale - m), row sum, row maximum
+      uint32_t pk[32];
+      float mx = -INFINITY, sum = 0.f;
 #pragma unroll
-      for (int c = 0; c < kBlockN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tS + lane_base + c * 32, r);
-        tmem_wait_ld();
-        uint32_t pk[16];
+      for (int j = 0; j < 16; ++j) {
+        const float a0 = __uint_as_float(r0[2 * j]), a1 = __uint_as_float(r0[2 * j + 1]);
+        mx = fmaxf(mx, fmaxf(a0, a1));
+        const float p0 = fast_exp2(fmaf(a0, scale_log2, -m_used));
+        const float p1 = fast_exp2(fmaf(a1, scale_log2, -m_used));
+        sum += p0;
+        sum += p1;
+        pk[j] = pack_bf16x2(p0, p1);
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float a0 = __uint_as_float(r1[2 * j]), a1 = __uint_as_float(r1[2 * j + 1]);
+        mx = fmaxf(mx, fmaxf(a0, a1));
+        const float p0 = fast_exp2(fmaf(a0, scale_log2, -m_used));
+        const float p1 = fast_exp2(fmaf(a1, scale_log2, -m_used));
+        sum += p0;
+        sum += p1;
+        pk[16 + j] = pack_bf16x2(p0, p1);
+      }
+      const float m_tile = mx * scale_log2;
+      const bool need = !(m_tile - m_used <= kRescaleThreshold);  // also true for the first tile (m = -inf)
+      if (__any_sync(0xffffffffu, need)) {
+        // rare path: adopt the new maximum for the rows that need it and redo the tile
+        float alpha = 1.f;
+        if (need) {
+          alpha = fast_exp2(m_used - m_tile);  // 0 on the first tile
+          m_used = m_tile;
+          l *= alpha;
+        }
+        sum = 0.f;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * j]), scale_log2, -m_used));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * j + 1]), scale_log2, -m_used));
-          if constexpr (!kSparse) {
-            if (c * 32 + 2 * j >= valid_cols) p0 = 0.f;
-            if (c * 32 + 2 * j + 1 >= valid_cols) p1 = 0.f;
-          }
+          const float p0 = fast_exp2(fmaf(__uint_as_float(r0[2 * j]), scale_log2, -m_used));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(r0[2 * j + 1]), scale_log2, -m_used));
           sum += p0;
           sum += p1;
           pk[j] = pack_bf16x2(p0, p1);
         }
-        tmem_st16(tS + lane_base + c * 16, pk);
-      }
-      l += sum;
-      if (any_need) {
-        // the previous P V finished before this tile's S was signalled, so O is quiescent
 #pragma unroll
-        for (int c = 0; c < kHeadDim / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tO + lane_base + c * 32, r);
-          tmem_wait_ld();
+        for (int j = 0; j < 16; ++j) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(r1[2 * j]), scale_log2, -m_used));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(r1[2 * j + 1]), scale_log2, -m_used));
+          sum += p0;
+          sum += p1;
+          pk[16 + j] = pack_bf16x2(p0, p1);
+        }
+        if (t > 0) {
+          // O must be quiescent: wait until P_{t-1} V_{t-1} has drained (its V stage was released)
+          const int tp = t - 1;
+          if (!mbar_wait(&sm.v_empty[tp % kStages], (tp / kStages) & 1, &sm.abort_flag, p.status, 32)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-          tmem_st32(tO + lane_base + c * 32, r);
+          for (int c = 0; c < kHeadDim / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + lane_base + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+            tmem_st32(tO + lane_base + c * 32, o);
+          }
         }
       }
+      l += sum;
+      tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&sm.p_full);
+      mbar_arrive(&sm.p_full[t & 1]);
     }
 
     // ---- epilogue: O / l -> bf16 -> global; LSE ----------------------------------------
@@ -293,11 +339,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int kBlockN, int kRowsQ, bool kSparse>
+template <bool kSparse, int kBlock, int kRowsQ>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kBlockN, kRowsQ, kSparse>;
-  const int smem = static_cast<int>(sizeof(AttnSmem<kBlockN>)) + 1024;
+  auto kernel = attn_kernel<kSparse, kBlock, kRowsQ>;
+  const int smem = static_cast<int>(sizeof(AttnSmem)) + 1024;
   static bool configured[64] = {};  // per template instantiation and device
   int dev = 0;
   cudaGetDevice(&dev);
@@ -314,15 +360,17 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
 
 }  // namespace
 
+// Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows.
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream) {
-  return launch<128, 128, false>(tq, tk, tv, p, batch, stream);
+  return launch<false, 128, 128>(tq, tk, tv, p, batch, stream);
 }
 
+// Tensor maps: Q box 64 x block_size rows, K and V boxes 64 x 64 rows.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128, 128, true>(tq, tk, tv, p, batch, stream);
-  return launch<64, 64, true>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<true, 128, 128>(tq, tk, tv, p, batch, stream);
+  return launch<true, 64, 64>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed
