@@ -3,8 +3,8 @@
 //
 // One CTA owns one query tile of one (batch, head) and streams 64-key tiles through a
 // warp-specialised pipeline:
-//   warp 4  : TMA producer  - Q once, then a K tile and a V tile per step into two-stage
-//                             rings of 128B-swizzled shared memory
+//   warp 4  : TMA producer  - Q once, then a K tile and a V tile per step into a five-slot
+//                             ring of 128B-swizzled shared memory shared by K and V
 //   warp 5  : UMMA issuer   - S_j = Q K_j^T into one of two tensor-memory buffers, then
 //                             O += P_j V_j with P read from tensor memory (P overwrites the
 //                             first half of S_j's columns). S_{j+1} is issued before P_j V_j,
@@ -15,7 +15,7 @@
 //             grew by more than 2^8 is the tile redone with the new maximum and O rescaled
 //             (after the previous P V has drained). Finally O is normalised and stored.
 // The dense kernel walks all key tiles; the sparse kernel walks the CSR list of its query
-// block (a 128-key block is two consecutive tiles). Two CTAs fit on one SM (96 KB of shared
+// block (a 128-key block is two consecutive tiles). Two CTAs fit on one SM (112 KB of shared
 // memory and 256 tensor-memory columns each).
 #include "internal.h"
 
@@ -25,7 +25,7 @@ namespace {
 constexpr int kHeadDim = 128;
 constexpr int kTileM = 128;   // UMMA M; rows of tensor memory
 constexpr int kTileN = 64;    // keys per pipeline step
-constexpr int kStages = 2;    // K and V ring depth
+constexpr int kSlots = 5;     // ring of 64-key tiles shared by K and V: load 2t is K_t, load 2t+1 is V_t
 constexpr int kSoftmaxThreads = 128;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
@@ -33,11 +33,20 @@ constexpr int kColS = 0;      // two S buffers of 64 fp32 columns; P (bf16 pairs
 constexpr int kColO = 128;    // O accumulator (fp32, 128 columns)
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
 
+// Debug builds (-DSPARSED_TIMELINE) record clock64 stamps of one CTA's pipeline roles after the
+// workspace status block: 3 regions of 2048 int64 (softmax thread 0, UMMA thread, TMA thread).
+#ifdef SPARSED_TIMELINE
+#define TL_DECL(region) long long* tl_buf = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(p.status) + 1024) + (region) * 2048; int tl_n = 0; const bool tl_on = (blockIdx.x == 1000) && ((threadIdx.x & 31) == 0);
+#define TL(tag) do { if (tl_on && tl_n < 2047) { tl_buf[1 + tl_n++] = (static_cast<long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFll); tl_buf[0] = tl_n; } } while (0)
+#else
+#define TL_DECL(region)
+#define TL(tag)
+#endif
+
 struct AttnSmem {
   alignas(1024) __nv_bfloat16 q[2][kTileM * 64];           // two 64-wide halves of head_dim
-  alignas(1024) __nv_bfloat16 k[kStages][2][kTileN * 64];
-  alignas(1024) __nv_bfloat16 v[kStages][2][kTileN * 64];
-  uint64_t q_full, k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  alignas(1024) __nv_bfloat16 kv[kSlots][2][kTileN * 64];  // each slot: two 64-wide halves of head_dim
+  uint64_t q_full, kv_full[kSlots], kv_empty[kSlots];
   uint64_t s_full[2], p_full[2], o_full;
   uint32_t tmem_base;
   int abort_flag;
@@ -49,8 +58,13 @@ template <bool kSparse, int kBlock, int kRowsQ>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  AttnSmem& sm = *reinterpret_cast<AttnSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  AttnSmem& sm = *reinterpret_cast<AttnSmem*>(smem_raw);
+  if ((smem_u32(smem_raw) & 1023u) != 0u) {
+    // swizzled tiles need a 1024-byte aligned base; never expected, reported instead of trusted
+    if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, 2) == 0) p.status->where = 1;
+    return;
+  }
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -77,11 +91,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // ---- set-up --------------------------------------------------------------------------
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.k_full[s], 1);
-      mbar_init(&sm.k_empty[s], 1);
-      mbar_init(&sm.v_full[s], 1);
-      mbar_init(&sm.v_empty[s], 1);
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(&sm.kv_full[s], 1);
+      mbar_init(&sm.kv_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.s_full[s], 1);
@@ -112,17 +124,24 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const uint32_t tmem = sm.tmem_base;
   const uint32_t tO = tmem + kColO;
 
+  // Warps 4 and 5 run their loops with all 32 lanes converged and let one elected lane issue
+  // the TMA / UMMA instructions: their operands then stay on the uniform datapath.
   if (warp == 4) {
     // =============================== TMA producer =======================================
-    if (lane == 0 && num_tiles > 0) {
-      tma_prefetch_desc(&tm_q);
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(&sm.q_full, kRowsQ * kHeadDim * 2);
-      tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
-      tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
+    if (num_tiles > 0) {
+      if (elect_one_sync()) {
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        mbar_expect_tx(&sm.q_full, kRowsQ * kHeadDim * 2);
+        tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
+        tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
+      }
+      __syncwarp();
       int block_id = 0;
-      for (int t = 0; t < num_tiles; ++t) {
+      TL_DECL(2)
+      bool ok = true;
+      for (int t = 0; ok && t < num_tiles; ++t) {
         int kv_row0;
         if constexpr (kSparse) {
           if (t % kTilesPerBlock == 0) block_id = __ldg(p.col_idx + list_begin + t / kTilesPerBlock);
@@ -130,62 +149,97 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         } else {
           kv_row0 = t * kTileN;
         }
-        const int s = t % kStages;
-        const int use = t / kStages;
-        if (use > 0 && !mbar_wait(&sm.k_empty[s], (use - 1) & 1, &sm.abort_flag, p.status, 10)) break;
-        mbar_expect_tx(&sm.k_full[s], kTileN * kHeadDim * 2);
-        tma_load_4d(sm.k[s][0], &tm_k, &sm.k_full[s], 0, kv_row0, kv_head, batch);
-        tma_load_4d(sm.k[s][1], &tm_k, &sm.k_full[s], 64, kv_row0, kv_head, batch);
-        if (use > 0 && !mbar_wait(&sm.v_empty[s], (use - 1) & 1, &sm.abort_flag, p.status, 11)) break;
-        mbar_expect_tx(&sm.v_full[s], kTileN * kHeadDim * 2);
-        tma_load_4d(sm.v[s][0], &tm_v, &sm.v_full[s], 0, kv_row0, kv_head, batch);
-        tma_load_4d(sm.v[s][1], &tm_v, &sm.v_full[s], 64, kv_row0, kv_head, batch);
+        // load 2t (K_t) and load 2t+1 (V_t); a slot is reused every kSlots loads
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+          const int i = 2 * t + which;
+          const int slot = i % kSlots;
+          TL(20 + which);
+          if (i >= kSlots) {
+            ok = mbar_wait(&sm.kv_empty[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          if (elect_one_sync()) {
+            mbar_expect_tx(&sm.kv_full[slot], kTileN * kHeadDim * 2);
+            const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+            tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
+            tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+          }
+          __syncwarp();
+        }
+        TL(22);
       }
     }
   } else if (warp == 5) {
     // =============================== UMMA issuer ========================================
-    if (lane == 0 && num_tiles > 0) {
+    if (num_tiles > 0) {
       constexpr uint32_t idesc_qk = umma_idesc_bf16(kTileM, kTileN, false, false);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(kTileM, kHeadDim, false, true);
-      const uint32_t q_addr[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
+      constexpr uint32_t hi_desc = umma_desc_hi_sw128(1024);
+      // descriptor low words: Q is fixed; K/V slots differ only in their base address
+      const uint32_t q_lo0 = umma_desc_lo(smem_u32(sm.q[0]), 16);
+      const uint32_t kv_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), 16);            // as K (K-major)
+      const uint32_t v_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), kTileN * 128);   // as V (MN-major)
+      constexpr uint32_t q_half_step = (kTileM * 64 * 2) >> 4;                    // 16 KB per head_dim half of Q
+      constexpr uint32_t slot_step = (2 * kTileN * 64 * 2) >> 4;                  // 16 KB per ring slot
+      constexpr uint32_t half_step = (kTileN * 64 * 2) >> 4;                      // 8 KB per head_dim half
+      TL_DECL(1)
       // S_t = Q K_t^T into S buffer t & 1
       auto issue_qk = [&](int t) -> bool {
-        const int s = t % kStages;
-        if (!mbar_wait(&sm.k_full[s], (t / kStages) & 1, &sm.abort_flag, p.status, 21)) return false;
+        const int i = 2 * t;
+        const int slot = i % kSlots;
+        TL(10);
+        bool got = mbar_wait(&sm.kv_full[slot], (i / kSlots) & 1, &sm.abort_flag, p.status, 21);
+        got = __all_sync(0xffffffffu, got);
+        if (!got) return false;
+        TL(11);
         tc_fence_after();
-        const uint32_t k_addr[2] = {smem_u32(sm.k[s][0]), smem_u32(sm.k[s][1])};
-        const uint32_t tS = tmem + kColS + (t & 1) * kTileN;
+        if (elect_one_sync()) {
+          const uint32_t k_lo = kv_lo0 + slot * slot_step;
+          const uint32_t tS = tmem + kColS + (t & 1) * kTileN;
+          umma_ss_words<false>(tS, q_lo0, hi_desc, k_lo, hi_desc, idesc_qk);
 #pragma unroll
-        for (int kk = 0; kk < kHeadDim / 16; ++kk) {
-          const uint32_t off = (kk & 3) * 32;
-          umma_ss(tS, umma_smem_desc_sw128(q_addr[kk >> 2] + off, 16, 1024),
-                  umma_smem_desc_sw128(k_addr[kk >> 2] + off, 16, 1024), idesc_qk, kk > 0);
+          for (int kk = 1; kk < kHeadDim / 16; ++kk) {
+            umma_ss_words<true>(tS, q_lo0 + (kk >> 2) * q_half_step + (kk & 3) * 2, hi_desc,
+                                k_lo + (kk >> 2) * half_step + (kk & 3) * 2, hi_desc, idesc_qk);
+          }
+          umma_commit(&sm.kv_empty[slot]);
+          umma_commit(&sm.s_full[t & 1]);
         }
-        umma_commit(&sm.k_empty[s]);
-        umma_commit(&sm.s_full[t & 1]);
+        __syncwarp();
+        TL(12);
         return true;
       };
       bool ok = mbar_wait(&sm.q_full, 0, &sm.abort_flag, p.status, 20);
+      ok = __all_sync(0xffffffffu, ok);
       ok = ok && issue_qk(0);
       for (int t = 0; ok && t < num_tiles; ++t) {
         // The S buffer of tile t+1 last held P_{t-1}, whose P V was issued one iteration ago,
         // and tcgen05 operations of one thread execute in issue order.
         if (t + 1 < num_tiles && !issue_qk(t + 1)) break;
-        const int s = t % kStages;
-        const uint32_t ph = (t >> 1) & 1;
-        if (!mbar_wait(&sm.p_full[t & 1], ph, &sm.abort_flag, p.status, 22)) break;
-        if (!mbar_wait(&sm.v_full[s], (t / kStages) & 1, &sm.abort_flag, p.status, 23)) break;
+        const int i = 2 * t + 1;
+        const int slot = i % kSlots;
+        ok = mbar_wait(&sm.p_full[t & 1], (t >> 1) & 1, &sm.abort_flag, p.status, 22);
+        TL(13);
+        ok = ok && mbar_wait(&sm.kv_full[slot], (i / kSlots) & 1, &sm.abort_flag, p.status, 23);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        TL(14);
         tc_fence_after();
-        const uint32_t v_addr = smem_u32(sm.v[s][0]);
-        const uint32_t tP = tmem + kColS + (t & 1) * kTileN;
+        if (elect_one_sync()) {
+          const uint32_t v_lo = v_lo0 + slot * slot_step;
+          const uint32_t tP = tmem + kColS + (t & 1) * kTileN;
+          // V tile is [key][d]: MN-major B operand; 16 keys per step are 2048 bytes apart
+          umma_ts_words(tO, tP, v_lo, hi_desc, idesc_pv, t > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < kTileN / 16; ++kk) {
-          // V tile is [key][d]: MN-major B operand; the two 64-wide d halves are kTileN*128 bytes apart
-          umma_ts(tO, tP + kk * 8, umma_smem_desc_sw128(v_addr + kk * 2048, kTileN * 128, 1024), idesc_pv,
-                  (t > 0) || (kk > 0));
+          for (int kk = 1; kk < kTileN / 16; ++kk)
+            umma_ts_words(tO, tP + kk * 8, v_lo + kk * 128, hi_desc, idesc_pv, 1u);
+          umma_commit(&sm.kv_empty[slot]);
+          if (t == num_tiles - 1) umma_commit(&sm.o_full);
         }
-        umma_commit(&sm.v_empty[s]);
-        if (t == num_tiles - 1) umma_commit(&sm.o_full);
+        __syncwarp();
+        TL(15);
       }
     }
   } else {
@@ -195,17 +249,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     float m_used = -INFINITY;
     float l = 0.f;
     bool ok = true;
+    TL_DECL(0)
+#ifdef SPARSED_TIMELINE
+    const bool tl_on2 = tl_on && tid == 0;
+#undef TL
+#define TL(tag) do { if (tl_on2 && tl_n < 2047) { tl_buf[1 + tl_n++] = (static_cast<long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFll); tl_buf[0] = tl_n; } } while (0)
+#endif
     for (int t = 0; t < num_tiles; ++t) {
+      TL(1);
       if (!mbar_wait(&sm.s_full[t & 1], (t >> 1) & 1, &sm.abort_flag, p.status, 30)) {
         ok = false;
         break;
       }
+      TL(2);
       tc_fence_after();
       const uint32_t tS = tmem + kColS + (t & 1) * kTileN + lane_base;
       uint32_t r0[32], r1[32];
       tmem_ld32(tS, r0);
       tmem_ld32(tS + 32, r1);
       tmem_wait_ld();
+      TL(3);
       if constexpr (!kSparse) {
         const int valid_cols = p.seq_len - t * kTileN;  // only the last tile can be ragged
         if (valid_cols < kTileN) {
@@ -268,8 +331,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         if (t > 0) {
           // O must be quiescent: wait until P_{t-1} V_{t-1} has drained (its V stage was released)
-          const int tp = t - 1;
-          if (!mbar_wait(&sm.v_empty[tp % kStages], (tp / kStages) & 1, &sm.abort_flag, p.status, 32)) {
+          const int ip = 2 * (t - 1) + 1;  // the load index of V_{t-1}
+          if (!mbar_wait(&sm.kv_empty[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
             ok = false;
             break;
           }
@@ -286,10 +349,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       }
       l += sum;
+      TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sm.p_full[t & 1]);
+      TL(5);
     }
 
     // ---- epilogue: O / l -> bf16 -> global; LSE ----------------------------------------
@@ -343,7 +408,7 @@ template <bool kSparse, int kBlock, int kRowsQ>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
   auto kernel = attn_kernel<kSparse, kBlock, kRowsQ>;
-  const int smem = static_cast<int>(sizeof(AttnSmem)) + 1024;
+  const int smem = static_cast<int>(sizeof(AttnSmem));
   static bool configured[64] = {};  // per template instantiation and device
   int dev = 0;
   cudaGetDevice(&dev);
