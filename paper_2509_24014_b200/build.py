@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsparsed.so")
 SOURCES = ["api.cu", "attention.cu", "scoring.cu", "topk.cu"]
-HEADERS = ["internal.h", "sm100_primitives.cuh", os.path.join("..", "..", "include", "sparsed.h")]
+HEADERS = ["internal.h", "sm100_primitives.cuh", "topk_device.cuh", os.path.join("..", "..", "include", "sparsed.h")]
 
 
 def _nvcc() -> str:

@@ -146,30 +146,38 @@ sparsed_status kept_counts(const sparsed_select_params* sp, int nb, int* pb, int
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-sparsed_status run_topk(const float* scores, int batch, int heads_q, int nb, int block_size, int pb, int k_pre,
-                        int k_gen, sparsed_pattern* out, cudaStream_t stream) {
+// Checks the caller's pattern buffers against the number of rows and kept blocks per row and
+// fills in the host-side fields of `out`.
+sparsed_status prepare_pattern(sparsed_pattern* out, int batch, int heads_q, int nb, int block_size, int k_total) {
   if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
-  if (nb > 1024) return SPARSED_ERR_UNSUPPORTED;
+  if (nb > 16384) return SPARSED_ERR_UNSUPPORTED;
   const int64_t rows = static_cast<int64_t>(batch) * heads_q * nb;
-  const int64_t nnz = rows * (k_pre + k_gen);
+  const int64_t nnz = rows * k_total;
   if (rows >= INT32_MAX || nnz >= INT32_MAX) return SPARSED_ERR_UNSUPPORTED;
   if (out->col_capacity < nnz) return SPARSED_ERR_PATTERN;
+  out->nnz = nnz;
+  out->block_size = block_size;
+  out->num_blocks = nb;
+  out->batch = batch;
+  out->heads_q = heads_q;
+  return SPARSED_OK;
+}
+
+sparsed_status run_topk(const float* scores, int batch, int heads_q, int nb, int block_size, int pb, int k_pre,
+                        int k_gen, sparsed_pattern* out, cudaStream_t stream) {
+  sparsed_status st = prepare_pattern(out, batch, heads_q, nb, block_size, k_pre + k_gen);
+  if (st != SPARSED_OK) return st;
   TopkParams tp;
   tp.scores = scores;
   tp.row_ptr = out->row_ptr;
   tp.col_idx = out->col_idx;
-  tp.rows = static_cast<int>(rows);
+  tp.rows = batch * heads_q * nb;
   tp.nb = nb;
   tp.pb = pb;
   tp.k_pre = k_pre;
   tp.k_gen = k_gen;
   cudaError_t e = launch_topk_csr(tp, stream);
   if (e != cudaSuccess) return cuda_fail(e);
-  out->nnz = nnz;
-  out->block_size = block_size;
-  out->num_blocks = nb;
-  out->batch = batch;
-  out->heads_q = heads_q;
   return SPARSED_OK;
 }
 
@@ -350,20 +358,23 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   if ((st = kept_counts(params, nb, &pb, &k_pre, &k_gen)) != SPARSED_OK) return st;
   if (q == nullptr || k == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k)) return SPARSED_ERR_ALIGNMENT;
-  if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
-  size_t need = 0;
-  if ((st = sparsed_workspace_bytes(SPARSED_OP_SELECT_PATTERN, shape, params, &need)) != SPARSED_OK) return st;
+  if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
+    return st;
+  // With few enough blocks per row the pooled-scoring kernel ranks each block-row in its own
+  // tail; A' then goes to memory only if the caller asked for it.
+  const bool fused = nb <= kFusedTopkMaxBlocks;
   const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
   const size_t score_bytes = round_up(bh * nb * nb * 4, 256);
   const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
-  size_t required = SPARSED_STATUS_BYTES + (scores_out_or_null ? 0 : score_bytes) + (lse_or_null ? 0 : lse_bytes);
+  const bool need_score_ws = !fused && scores_out_or_null == nullptr;
+  const size_t required = SPARSED_STATUS_BYTES + (need_score_ws ? score_bytes : 0) + (lse_or_null ? 0 : lse_bytes);
   if (ws == nullptr || ws_bytes < required) return SPARSED_ERR_WORKSPACE;
   if ((st = check_arch()) != SPARSED_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* base = static_cast<uint8_t*>(ws);
   float* scores = scores_out_or_null;
   size_t off = SPARSED_STATUS_BYTES;
-  if (scores == nullptr) {
+  if (need_score_ws) {
     scores = reinterpret_cast<float*>(base + off);
     off += score_bytes;
   }
@@ -379,6 +390,11 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   sp.block_size = params->block_size;
   sp.scale_log2 = rs.scale_log2;
   sp.status = static_cast<DeviceStatus*>(ws);
+  sp.row_ptr = fused ? out->row_ptr : nullptr;
+  sp.col_idx = fused ? out->col_idx : nullptr;
+  sp.pb = pb;
+  sp.k_pre = k_pre;
+  sp.k_gen = k_gen;
   if (lse_or_null == nullptr) {
     float* lse_buf = reinterpret_cast<float*>(base + off);
     cudaError_t e = launch_row_stats(tq, tk, sp, lse_buf, shape->batch, stream);
@@ -387,6 +403,7 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   }
   cudaError_t e = launch_pooled_scores(tq, tk, sp, shape->batch, stream);
   if (e != cudaSuccess) return cuda_fail(e);
+  if (fused) return SPARSED_OK;
   return run_topk(scores, shape->batch, shape->heads_q, nb, params->block_size, pb, k_pre, k_gen, out, stream);
 }
 

@@ -11,9 +11,10 @@
 //                             so the tensor pipe works on the next logits while the softmax
 //                             warps are busy with the current ones.
 //   warps 0-3: one thread per query row - online softmax in fp32 on base-2 logits. The tile
-//             is exponentiated once against the running maximum; only if some row's maximum
-//             grew by more than 2^8 is the tile redone with the new maximum and O rescaled
-//             (after the previous P V has drained). Finally O is normalised and stored.
+//             is exponentiated once against the running maximum; only if a row sum shows that
+//             logits may have outgrown it by more than 2^8 is the tile redone with the new
+//             maximum and O rescaled (after the previous P V has drained). Finally O is
+//             normalised and stored.
 // The dense kernel walks all key tiles; the sparse kernel walks the CSR list of its query
 // block (a 128-key block is two consecutive tiles). Two CTAs fit on one SM (112 KB of shared
 // memory and 256 tensor-memory columns each).
@@ -31,7 +32,10 @@ constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0;      // two S buffers of 64 fp32 columns; P (bf16 pairs) reuses the first 32
 constexpr int kColO = 128;    // O accumulator (fp32, 128 columns)
-constexpr float kRescaleThreshold = 8.0f;  // in log2 units
+#ifndef SPARSED_ATTN_POLY_EVERY
+#define SPARSED_ATTN_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = SPARSED_ATTN_POLY_EVERY;  // every n-th exponential on the FMA pipes (0 = none)
 
 // Debug builds (-DSPARSED_TIMELINE) record clock64 stamps of one CTA's pipeline roles after the
 // workspace status block: 3 regions of 2048 int64 (softmax thread 0, UMMA thread, TMA thread).
@@ -279,35 +283,38 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
         }
       }
-      // one pass against the running maximum: p = 2^(s*scale - m), row sum, row maximum
+      // Fast path: one pass against the running maximum m, p = 2^(s*scale - m), with packed
+      // fp32x2 arithmetic. No row maximum is taken here: if every p were above 2^8 the row sum
+      // would exceed 2^8 too, so a sum <= 2^8 proves that the stale maximum is still safe.
       uint32_t pk[32];
-      float mx = -INFINITY, sum = 0.f;
+      float sum;
+      {
+        const float2 sc = make_float2(scale_log2, scale_log2);
+        const float2 nm = make_float2(-m_used, -m_used);
+        float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float a0 = __uint_as_float(r0[2 * j]), a1 = __uint_as_float(r0[2 * j + 1]);
-        mx = fmaxf(mx, fmaxf(a0, a1));
-        const float p0 = fast_exp2(fmaf(a0, scale_log2, -m_used));
-        const float p1 = fast_exp2(fmaf(a1, scale_log2, -m_used));
-        sum += p0;
-        sum += p1;
-        pk[j] = pack_bf16x2(p0, p1);
+        for (int j = 0; j < 16; ++j) {
+          const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(r0[2 * j]), __uint_as_float(r0[2 * j + 1])), sc, nm);
+          const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(r1[2 * j]), __uint_as_float(r1[2 * j + 1])), sc, nm);
+          const float2 e0 = make_float2(tile_exp2<kPolyEvery>(x0.x, 2 * j), tile_exp2<kPolyEvery>(x0.y, 2 * j + 1));
+          const float2 e1 = make_float2(tile_exp2<kPolyEvery>(x1.x, 2 * j), tile_exp2<kPolyEvery>(x1.y, 2 * j + 1));
+          acc0 = __fadd2_rn(acc0, e0);
+          acc1 = __fadd2_rn(acc1, e1);
+          pk[j] = pack_bf16x2(e0.x, e0.y);
+          pk[16 + j] = pack_bf16x2(e1.x, e1.y);
+        }
+        sum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
       }
+      const bool trigger = !(sum <= 256.0f);  // also true on the first tile (m = -inf) and for NaN
+      if (__any_sync(0xffffffffu, trigger)) {
+        // Slow path (first tile, or logits that outgrew the running maximum): take the true row
+        // maximum, adopt it where it grew, redo the tile and rescale what O holds so far.
+        float mx = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float a0 = __uint_as_float(r1[2 * j]), a1 = __uint_as_float(r1[2 * j + 1]);
-        mx = fmaxf(mx, fmaxf(a0, a1));
-        const float p0 = fast_exp2(fmaf(a0, scale_log2, -m_used));
-        const float p1 = fast_exp2(fmaf(a1, scale_log2, -m_used));
-        sum += p0;
-        sum += p1;
-        pk[16 + j] = pack_bf16x2(p0, p1);
-      }
-      const float m_tile = mx * scale_log2;
-      const bool need = !(m_tile - m_used <= kRescaleThreshold);  // also true for the first tile (m = -inf)
-      if (__any_sync(0xffffffffu, need)) {
-        // rare path: adopt the new maximum for the rows that need it and redo the tile
+        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fmaxf(__uint_as_float(r0[j]), __uint_as_float(r1[j])));
+        const float m_tile = mx * scale_log2;
         float alpha = 1.f;
-        if (need) {
+        if (m_tile > m_used) {
           alpha = fast_exp2(m_used - m_tile);  // 0 on the first tile
           m_used = m_tile;
           l *= alpha;
@@ -330,7 +337,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           pk[16 + j] = pack_bf16x2(p0, p1);
         }
         if (t > 0) {
-          // O must be quiescent: wait until P_{t-1} V_{t-1} has drained (its V stage was released)
+          // O must be quiescent: wait until P_{t-1} V_{t-1} has drained (its ring slot was released)
           const int ip = 2 * (t - 1) + 1;  // the load index of V_{t-1}
           if (!mbar_wait(&sm.kv_empty[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
             ok = false;

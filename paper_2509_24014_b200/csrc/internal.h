@@ -26,7 +26,7 @@ struct AttnParams {
 
 // Parameters of the pooled-scoring kernel.
 struct ScoreParams {
-  float* scores;           // fp32 [B,Hq,nb,nb]
+  float* scores;           // fp32 [B,Hq,nb,nb], or null when only the pattern is wanted (fused top-k)
   const float* lse;        // fp32 [B,Hq,L], natural log
   int seq_len;
   int heads_q;
@@ -34,7 +34,14 @@ struct ScoreParams {
   int block_size;          // 64 or 128
   float scale_log2;
   DeviceStatus* status;
+  // fused selection (row_ptr != null): each CTA ranks the block-row(s) it has just pooled
+  int32_t* row_ptr;
+  int32_t* col_idx;
+  int pb, k_pre, k_gen;
 };
+
+// Largest number of key blocks per row the pooled-scoring kernel can rank in its own tail.
+constexpr int kFusedTopkMaxBlocks = 1024;
 
 struct TopkParams {
   const float* scores;     // fp32 [rows, nb]

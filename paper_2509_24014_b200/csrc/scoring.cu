@@ -10,7 +10,11 @@
 // Pipeline per CTA: warp 4 streams K tiles by TMA (two stages), warp 5 issues S = Q K^T
 // into one of two tensor-memory buffers, warps 0-3 (one thread per query row) exponentiate
 // and reduce. Sums run in a fixed order, so results are bitwise reproducible.
+// With a pattern to fill (row_ptr != null) warp 0 also keeps the block-row(s) it produced as
+// ordered keys in shared memory and, after the last tile, runs the isolated top-k of Eq. 5/6
+// on them and writes the CSR lists: selection then needs no pass over A' in memory.
 #include "internal.h"
+#include "topk_device.cuh"
 
 namespace sparsed {
 namespace {
@@ -26,6 +30,8 @@ struct ScoreSmem {
   alignas(1024) __nv_bfloat16 k[kStages][2][kTile * 64];
   uint64_t q_full, k_full[kStages], k_empty[kStages], s_full[2], s_empty[2], partial_full[4];
   float partial[4][4][2];  // [tile % 4][warp][column half]
+  uint32_t keys[2][kFusedTopkMaxBlocks];  // ordered keys of the block-row(s) of this CTA (fused top-k)
+  int hist[256];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -34,8 +40,12 @@ template <bool kStatsOnly>
 __global__ void __launch_bounds__(kThreads, 2)
 score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
              const ScoreParams p, float* lse_out) {
-  extern __shared__ uint8_t smem_raw[];
-  ScoreSmem& sm = *reinterpret_cast<ScoreSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  ScoreSmem& sm = *reinterpret_cast<ScoreSmem*>(smem_raw);
+  if ((smem_u32(smem_raw) & 1023u) != 0u) {
+    if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, 2) == 0) p.status->where = 2;
+    return;
+  }
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   const int num_q_tiles = (p.seq_len + kTile - 1) / kTile;
@@ -122,6 +132,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     const int nb = p.seq_len / p.block_size;
     const bool half_blocks = (p.block_size == 64);
     const float inv_area = 1.f / (static_cast<float>(p.block_size) * static_cast<float>(p.block_size));
+    const bool fuse_topk = (!kStatsOnly) && (p.row_ptr != nullptr);
     bool ok = true;
     for (int it = 0; it < num_tiles; ++it) {
       const int buf = it & 1;
@@ -195,18 +206,45 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (lane == 0) {
               const float* pp = &sm.partial[slot][0][0];
               const float total = ((pp[0] + pp[1]) + (pp[2] + pp[3])) + ((pp[4] + pp[5]) + (pp[6] + pp[7]));
-              p.scores[(static_cast<int64_t>(bh) * nb + q_tile) * nb + it] = total * inv_area;
+              const float score = total * inv_area;
+              if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + q_tile) * nb + it] = score;
+              if (fuse_topk) sm.keys[0][it] = ordered_key(score);
             }
           } else {
             const int rh = lane >> 1, ch = lane & 1;  // row half (warps 2rh, 2rh+1), column half
             const int ib = q_tile * 2 + rh, jb = it * 2 + ch;
             if (ib < nb && jb < nb) {
               const float total = sm.partial[slot][2 * rh][ch] + sm.partial[slot][2 * rh + 1][ch];
-              p.scores[(static_cast<int64_t>(bh) * nb + ib) * nb + jb] = total * inv_area;
+              const float score = total * inv_area;
+              if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + ib) * nb + jb] = score;
+              if (fuse_topk) sm.keys[rh][jb] = ordered_key(score);
             }
           }
         }
         __syncwarp();
+      }
+    }
+    if constexpr (!kStatsOnly) {
+      if (fuse_topk && warp == 0) {
+        // warp 0 wrote every key of this CTA's block-row(s); rank them now (Eq. 5 / Eq. 6)
+        const bool all_ok = __all_sync(0xffffffffu, ok);
+        __syncwarp();
+        if (all_ok) {
+          const int k_total = p.k_pre + p.k_gen;
+          const int rows_here = half_blocks ? 2 : 1;
+          for (int rh = 0; rh < rows_here; ++rh) {
+            const int ib = half_blocks ? q_tile * 2 + rh : q_tile;
+            if (ib >= nb) break;
+            const int64_t row = static_cast<int64_t>(bh) * nb + ib;
+            warp_select_row(sm.keys[rh], nb, p.pb, p.k_pre, p.k_gen, sm.hist, p.col_idx + row * k_total, lane);
+            if (lane == 0) {
+              p.row_ptr[row] = static_cast<int32_t>(row * k_total);
+              if (row == static_cast<int64_t>(gridDim.x / num_q_tiles) * nb - 1)
+                p.row_ptr[row + 1] = static_cast<int32_t>((row + 1) * k_total);
+            }
+            __syncwarp();
+          }
+        }
       }
     }
     if constexpr (kStatsOnly) {
@@ -226,7 +264,7 @@ template <bool kStatsOnly>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, float* lse_out, int batch,
                    cudaStream_t stream) {
   auto kernel = score_kernel<kStatsOnly>;
-  const int smem = static_cast<int>(sizeof(ScoreSmem)) + 1024;
+  const int smem = static_cast<int>(sizeof(ScoreSmem));
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   const int num_q_tiles = (p.seq_len + kTile - 1) / kTile;

@@ -312,4 +312,28 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// 2^x on the FMA and integer pipes instead of the special-function unit, for spreading the
+// exponentials of a softmax tile over both: x is split into floor(x) (taken from the low
+// mantissa bits of x + 1.5*2^23 rounded down) and a fraction in [0,1) whose power of two is a
+// degree-4 minimax polynomial (relative error 2.7e-6); the integer part is then added to the
+// exponent field. Valid for x <= 127; anything below -126 returns about 2^-126.
+__device__ __forceinline__ float poly_exp2(float x) {
+  x = fmaxf(x, -126.0f);
+  float t;
+  asm("add.rm.ftz.f32 %0, %1, %2;" : "=f"(t) : "f"(x), "f"(12582912.0f));
+  const float f = x - (t - 12582912.0f);
+  float pl = fmaf(0.013534167781472206f, f, 0.052011460065841675f);
+  pl = fmaf(pl, f, 0.2414427548646927f);
+  pl = fmaf(pl, f, 0.6930038332939148f);
+  pl = fmaf(pl, f, 1.0000026226043701f);
+  return __int_as_float(__float_as_int(pl) + (__float_as_int(t) << 23));
+}
+
+// Exponential of element j of a row: every kPolyEvery-th element goes to the polynomial.
+template <int kPolyEvery>
+__device__ __forceinline__ float tile_exp2(float x, int j) {
+  if (kPolyEvery > 0 && (j % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery - 1)) return poly_exp2(x);
+  return fast_exp2(x);
+}
+
 }  // namespace sparsed

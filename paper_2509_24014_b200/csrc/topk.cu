@@ -1,97 +1,41 @@
 // Per-row isolated top-k over pooled block scores and compaction into CSR block lists
-// (Eq. 5 / Eq. 6; the IndexSelection and mask-write lines of Algorithm 1).
+// (Eq. 5 / Eq. 6; the IndexSelection and mask-write lines of Algorithm 1), as a kernel of
+// its own for scores that already sit in memory.
 //
 // One warp owns one row (batch, head, query block) of A'. The row's nb fp32 scores are read
-// once, coalesced, into registers as order-preserving 32-bit keys. For each key region
-// (prefill blocks [0,pb), generation blocks [pb,nb)) the k-th largest key is found by a
-// 32-step bitwise search with warp-wide counts; blocks above it are kept, blocks equal to
-// it are kept lowest index first until k are kept (ties -> lower block index). Kept ids are
-// written in ascending order through ballot prefix sums. Every row keeps the same number of
-// blocks, so row_ptr is an arithmetic sequence written by the same kernel.
-// HBM-bound by design: 4*nb bytes read and 4*(k_pre+k_gen) + 4 bytes written per row.
+// once with coalesced 16-byte loads and parked in shared memory as order-preserving keys;
+// the selection itself is warp_select_row (radix selection + ordered ballot compaction).
+// Every row keeps the same number of blocks, so row_ptr is an arithmetic sequence written by
+// the same kernel. HBM-bound by design: 4*nb bytes read and 4*(k_pre+k_gen) + 4 bytes
+// written per row.
 #include "internal.h"
+#include "topk_device.cuh"
 
 namespace sparsed {
 namespace {
 
-// Order-preserving map float -> uint32 (larger float -> larger key). NaN ranks lowest,
-// -0 equals +0.
-__device__ __forceinline__ uint32_t ordered_key(float f) {
-  uint32_t u = __float_as_uint(f);
-  if ((u & 0x7fffffffu) > 0x7f800000u) return 0u;  // NaN
-  if (u == 0x80000000u) u = 0u;                    // -0 -> +0
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-template <int kSlots>
-__global__ void __launch_bounds__(256) topk_csr_kernel(const TopkParams p) {
-  const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+__global__ void __launch_bounds__(256) topk_csr_kernel(const TopkParams p, int warps_per_cta) {
+  extern __shared__ __align__(16) uint8_t topk_smem[];
+  const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  if (warp_global >= p.rows) return;
-  const int row = warp_global;
+  const int row = blockIdx.x * warps_per_cta + warp;
+  if (warp >= warps_per_cta || row >= p.rows) return;
+  const int nb_pad = (p.nb + 3) & ~3;
+  uint32_t* keys = reinterpret_cast<uint32_t*>(topk_smem) + static_cast<size_t>(warp) * (nb_pad + 256);
+  int* hist = reinterpret_cast<int*>(keys + nb_pad);
   const float* src = p.scores + static_cast<int64_t>(row) * p.nb;
+  if ((p.nb & 3) == 0) {
+    const float4* src4 = reinterpret_cast<const float4*>(src);
+    for (int i = lane; i < p.nb / 4; i += 32) {
+      const float4 v = __ldg(src4 + i);
+      reinterpret_cast<uint4*>(keys)[i] = make_uint4(ordered_key(v.x), ordered_key(v.y), ordered_key(v.z), ordered_key(v.w));
+    }
+  } else {
+    for (int i = lane; i < p.nb; i += 32) keys[i] = ordered_key(__ldg(src + i));
+  }
+  __syncwarp();
   const int k_total = p.k_pre + p.k_gen;
-
-  uint32_t key[kSlots];
-#pragma unroll
-  for (int t = 0; t < kSlots; ++t) {
-    const int idx = t * 32 + lane;
-    key[t] = (idx < p.nb) ? ordered_key(__ldg(src + idx)) : 0u;
-  }
-
-  uint32_t keep_mask = 0;  // bit t: this lane's slot t is kept (kSlots <= 32)
-#pragma unroll 1
-  for (int region = 0; region < 2; ++region) {
-    const int lo = region == 0 ? 0 : p.pb;
-    const int hi = region == 0 ? p.pb : p.nb;
-    const int kk = region == 0 ? p.k_pre : p.k_gen;
-    if (hi <= lo || kk <= 0) continue;
-    uint32_t in_region = 0;
-#pragma unroll
-    for (int t = 0; t < kSlots; ++t) {
-      const int idx = t * 32 + lane;
-      if (idx >= lo && idx < hi) in_region |= (1u << t);
-    }
-    // largest T with count(key >= T) >= kk  ==  the kk-th largest key of the region
-    uint32_t thr = 0;
-#pragma unroll 1
-    for (int bit = 31; bit >= 0; --bit) {
-      const uint32_t cand = thr | (1u << bit);
-      int cnt = 0;
-#pragma unroll
-      for (int t = 0; t < kSlots; ++t) cnt += ((in_region >> t) & 1u) && (key[t] >= cand);
-      cnt = __reduce_add_sync(0xffffffffu, cnt);
-      if (cnt >= kk) thr = cand;
-    }
-    int n_gt = 0;
-#pragma unroll
-    for (int t = 0; t < kSlots; ++t) n_gt += ((in_region >> t) & 1u) && (key[t] > thr);
-    n_gt = __reduce_add_sync(0xffffffffu, n_gt);
-    const int need_eq = kk - n_gt;  // >= 1
-    int eq_before = 0;              // equal keys at lower block indices (slot-major = index order)
-    const uint32_t lt_mask = (1u << lane) - 1u;
-#pragma unroll
-    for (int t = 0; t < kSlots; ++t) {
-      const bool in_r = (in_region >> t) & 1u;
-      const bool eq = in_r && (key[t] == thr);
-      const uint32_t b = __ballot_sync(0xffffffffu, eq);
-      const int rank = eq_before + __popc(b & lt_mask);
-      if (in_r && (key[t] > thr || (eq && rank < need_eq))) keep_mask |= (1u << t);
-      eq_before += __popc(b);
-    }
-  }
-
-  // ordered compaction: block ids ascending
-  int32_t* dst = p.col_idx + static_cast<int64_t>(row) * k_total;
-  int run = 0;
-  const uint32_t lt_mask = (1u << lane) - 1u;
-#pragma unroll
-  for (int t = 0; t < kSlots; ++t) {
-    const bool kp = (keep_mask >> t) & 1u;
-    const uint32_t b = __ballot_sync(0xffffffffu, kp);
-    if (kp) dst[run + __popc(b & lt_mask)] = t * 32 + lane;
-    run += __popc(b);
-  }
+  warp_select_row(keys, p.nb, p.pb, p.k_pre, p.k_gen, hist, p.col_idx + static_cast<int64_t>(row) * k_total, lane);
   if (lane == 0) {
     p.row_ptr[row] = row * k_total;
     if (row == p.rows - 1) p.row_ptr[p.rows] = p.rows * k_total;
@@ -122,17 +66,17 @@ __global__ void pattern_validate_kernel(const int32_t* row_ptr, const int32_t* c
 
 cudaError_t launch_topk_csr(const TopkParams& p, cudaStream_t stream) {
   if (p.rows <= 0) return cudaSuccess;
-  const int threads = 256;
-  const int warps_per_cta = threads / 32;
-  const unsigned ctas = static_cast<unsigned>((p.rows + warps_per_cta - 1) / warps_per_cta);
-  const int slots = (p.nb + 31) / 32;
-  if (slots <= 1) topk_csr_kernel<1><<<ctas, threads, 0, stream>>>(p);
-  else if (slots <= 2) topk_csr_kernel<2><<<ctas, threads, 0, stream>>>(p);
-  else if (slots <= 4) topk_csr_kernel<4><<<ctas, threads, 0, stream>>>(p);
-  else if (slots <= 8) topk_csr_kernel<8><<<ctas, threads, 0, stream>>>(p);
-  else if (slots <= 16) topk_csr_kernel<16><<<ctas, threads, 0, stream>>>(p);
-  else if (slots <= 32) topk_csr_kernel<32><<<ctas, threads, 0, stream>>>(p);
-  else return cudaErrorInvalidValue;
+  if (p.nb > 16384) return cudaErrorInvalidValue;
+  const int warps = p.nb <= 1024 ? 8 : (p.nb <= 4096 ? 4 : 2);
+  const int nb_pad = (p.nb + 3) & ~3;
+  const size_t smem = static_cast<size_t>(warps) * (nb_pad + 256) * 4;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(topk_csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+  }
+  const unsigned ctas = static_cast<unsigned>((p.rows + warps - 1) / warps);
+  topk_csr_kernel<<<ctas, warps * 32, smem, stream>>>(p, warps);
   return cudaGetLastError();
 }
 
