@@ -346,11 +346,41 @@ def run_ours(args, cfg):
                 "frac_of_sustained": ach / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
                 "avg_launch_ms": ms, "traffic": NCU_DRAM_TRAFFIC.get((name, cfg.name))}
 
+    def topk_roofline():
+        """The ranking/compaction kernel alone (sparsed_select_from_scores) on this workload's A',
+        HBM-bound by design; L2 is flushed before each launch by writing a 512 MB buffer."""
+        scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=dev)
+        sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse, scores_out=scores, shape=shape_qk)
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        pat2, rp2, ci2 = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+        times = []
+        for _ in range(5):
+            flush.fill_(1)
+            a, b = ev(), ev()
+            a.record()
+            sd.sparsed_select_from_scores(scores, params, pat2, ws)
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        assert torch.equal(ci2, col_idx) and torch.equal(rp2, row_ptr)
+        ms = min(times[1:])
+        nbytes = B * Hq * (4 * nb * nb + 4 * nb * (k_pre + k_gen) + 4 * nb)
+        ach = nbytes / (ms * 1e-3) / 1e9
+        return {"kernel": "topk_csr_kernel (stand-alone, not in the step)", "bound": "hbm", "achieved": ach,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                "peak_source": f"HBM copy, {tag}", "avg_launch_ms": ms, "algorithmic_bytes": nbytes,
+                "traffic": NCU_DRAM_TRAFFIC.get(("topk_csr_kernel", cfg.name)),
+                "note": "event time of a single launch includes launch latency; L2 flushed before it"}
+
     roof_dense = tensor_roofline("attn_kernel<dense>", dense_flops(cfg), full_ms)
     roof_sparse = tensor_roofline("attn_kernel<sparse>", sparse_flops(cfg, nnz), sparse_ms)
     # selection = pooled-scoring kernel (a dense QK^T contraction, 2*L^2*D per head) + top-k/CSR kernel
-    roof_select = tensor_roofline("score_kernel+topk_csr_kernel", dense_flops(cfg) / 2, select_ms)
+    fused_topk = nb <= 1024   # the scoring kernel ranks its own block-rows up to 1024 blocks per row
+    launches_per_step = 3 if fused_topk else 4
+    roof_select = tensor_roofline("score_kernel", dense_flops(cfg) / 2, select_ms)
+    roof_topk = topk_roofline()
     dominant = max((roof_dense, roof_select, roof_sparse), key=lambda r: r["avg_launch_ms"])
+    roof_all = [roof_dense, roof_select, roof_topk, roof_sparse]
 
     # ---- CPU oracle beside it (bounded sample of the same workload) ----------------------
     cpu = None
@@ -378,18 +408,49 @@ def run_ours(args, cfg):
         "dense_tflops": dense_tflops,
         "speedup_vs_dense": full_total / sparse_total, "ideal_speedup": nb / (k_pre + k_gen),
         "phase_ms": {"attn_full": full_total / n, "select_pattern": select_total / n, "attn_sparse": sparse_total / n},
-        "roofline": dominant, "roofline_by_kernel": [roof_dense, roof_select, roof_sparse],
+        "roofline": dominant, "roofline_by_kernel": roof_all,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "pinned host Q,K,V -> device, sparsed_attn_sparse, O -> pinned host", "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": 4 * n, "launches_per_step": {"attn_kernel<dense>": 1, "score_kernel": 1,
-                                                     "topk_csr_kernel": 1, "attn_kernel<sparse>": 1},
+        "gpu_launches": launches_per_step * n,
+        "launches_per_step": {"attn_kernel<dense>": 1, "score_kernel (pooled scoring + fused top-k/CSR)": 1,
+                              "topk_csr_kernel": 0 if fused_topk else 1, "attn_kernel<sparse>": 1},
         "clocks": clocks, "peaks": peaks,
     }
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_topk_only(args, cfg):
+    """The ranking/compaction kernel alone on seeded pseudo scores of this workload's shape
+    ([B,Hq,nb,nb] fp32): a small-footprint run for profiling that kernel by itself."""
+    import paper_2509_24014_b200 as sd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    B, Hq, nb = cfg.batch, cfg.heads_q, cfg.num_blocks
+    scores = syn.random_scores(B * Hq * nb, nb, seed=cfg.seed, device=dev).view(B, Hq, nb, nb)
+    params = sd.make_params(cfg.block_size, cfg.keep_ratio, cfg.prefill_len)
+    k_pre, k_gen = sd.sparsed_kept_per_row(params, cfg.seq_len)
+    pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+    ws = sd.new_workspace(256, dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    times = []
+    for _ in range(args.warmup + args.steps):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        sd.sparsed_select_from_scores(scores, params, pat, ws)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    ms = statistics.median(times[args.warmup:])
+    nbytes = B * Hq * (4 * nb * nb + 4 * nb * (k_pre + k_gen) + 4 * nb)
+    print(json.dumps({"kernel": "topk_csr_kernel", "workload": workload_name(cfg), "rows": B * Hq * nb, "nb": nb,
+                      "ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6,
+                      "frac_of_hbm_peak": nbytes / ms / 1e6 / peaks["hbm_gbs"], "l2": "flushed before each launch"}))
 
 
 def main():
@@ -402,9 +463,12 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=160, help="row blocks the CPU oracle is timed on")
     ap.add_argument("--ref-rows", type=int, default=4, help="row blocks per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only-topk", action="store_true", help="run only the stand-alone ranking kernel")
     args = ap.parse_args()
     cfg = syn.CONFIGS[args.config]
-    if args.impl == "reference":
+    if args.only_topk:
+        run_topk_only(args, cfg)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)

@@ -24,6 +24,10 @@ constexpr int kTile = 128;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
 constexpr int kStages = 2;
+#ifndef SPARSED_SCORE_POLY_EVERY
+#define SPARSED_SCORE_POLY_EVERY 0
+#endif
+constexpr int kScorePolyEvery = SPARSED_SCORE_POLY_EVERY;  // every n-th exponential on the FMA pipes (0 = none)
 
 struct ScoreSmem {
   alignas(1024) __nv_bfloat16 q[2][kTile * 64];
@@ -180,7 +184,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           tmem_wait_ld();
           float acc = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc += fast_exp2(fmaf(__uint_as_float(r[j]), scale_log2, -lse2));
+          for (int j = 0; j < 32; ++j)
+            acc += tile_exp2<kScorePolyEvery>(fmaf(__uint_as_float(r[j]), scale_log2, -lse2), j);
           half_sum[c >> 1] += acc;
         }
         tc_fence_before();

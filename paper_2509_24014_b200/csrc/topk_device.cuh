@@ -4,10 +4,11 @@
 //
 // For each key region (prefill blocks [0,pb), generation blocks [pb,nb)) the k-th largest key
 // is found by radix selection, 8 bits per pass over a 256-bin warp histogram in shared
-// memory, starting below the bits all keys of the region have in common; a pass is skipped
-// once the surviving bucket is exactly as large as the number still to take. Blocks above
-// the threshold are kept, blocks equal to it lowest index first (ties -> lower block index).
-// Kept ids are written in ascending order through ballot prefix sums.
+// memory, starting below the bits all keys of the region have in common. The search stops as
+// soon as the surviving bucket is exactly as large as the number still to take, and once the
+// bucket fits in a warp (<= 32 keys) it is finished by ranking those keys against each other.
+// Blocks above the threshold are kept, blocks equal to it lowest index first (ties -> lower
+// block index). Kept ids are written in ascending order through ballot prefix sums.
 #pragma once
 
 #include <stdint.h>
@@ -109,6 +110,40 @@ __device__ __forceinline__ RegionThreshold warp_region_threshold(const uint32_t*
     top = shift;
     if (bucket == need) break;  // the whole surviving bucket is kept: lower bits do not matter
     __syncwarp();
+    if (bucket <= 32 && top > 0) {
+      // Finish inside the warp: pull the bucket's keys into lanes (in index order) and rank them.
+      uint32_t* cand = reinterpret_cast<uint32_t*>(hist);
+      const uint32_t lt_mask = (1u << lane) - 1u;
+      int filled = 0;
+      for (int base = lo; base < hi; base += 32) {
+        const int i = base + lane;
+        uint32_t k = 0u;
+        bool in_bucket = false;
+        if (i < hi) {
+          k = keys[i];
+          in_bucket = (k & r.mask) == r.prefix;
+        }
+        const uint32_t b = __ballot_sync(0xffffffffu, in_bucket);
+        if (in_bucket) cand[filled + __popc(b & lt_mask)] = k;
+        filled += __popc(b);
+      }
+      __syncwarp();
+      const bool have = lane < bucket;
+      const uint32_t mine_key = have ? cand[lane] : 0u;
+      int rank = 0;  // keys ahead of mine in (key descending, position ascending) order
+      for (int j = 0; j < bucket; ++j) {
+        const uint32_t kj = __shfl_sync(0xffffffffu, mine_key, j);
+        rank += (kj > mine_key) || (kj == mine_key && j < lane);
+      }
+      const uint32_t pick = __ballot_sync(0xffffffffu, have && rank == need - 1);
+      const uint32_t thr = __shfl_sync(0xffffffffu, mine_key, __ffs(pick) - 1);
+      const int greater = __popc(__ballot_sync(0xffffffffu, have && mine_key > thr));
+      r.prefix = thr;
+      r.mask = 0xffffffffu;
+      need -= greater;
+      __syncwarp();
+      break;
+    }
   }
   r.take_equal = need;
   return r;
@@ -124,26 +159,31 @@ __device__ __forceinline__ void warp_select_row(const uint32_t* keys, int nb, in
   th[1] = warp_region_threshold(keys, pb, nb, k_gen, hist, lane);
   const uint32_t lt_mask = (1u << lane) - 1u;
   int run = 0;
-  int eq_seen[2] = {0, 0};
+  int eq_seen0 = 0, eq_seen1 = 0;
   for (int base = 0; base < nb; base += 32) {
     const int i = base + lane;
+    const bool second = i >= pb;  // which region this lane's block is in
+    const uint32_t mask = second ? th[1].mask : th[0].mask;
+    const uint32_t prefix = second ? th[1].prefix : th[0].prefix;
     bool keep = false, eq = false;
-    int region = 0;
     if (i < nb) {
-      region = i >= pb ? 1 : 0;
-      const uint32_t km = keys[i] & th[region].mask;
-      eq = km == th[region].prefix;
-      keep = km > th[region].prefix;
+      const uint32_t km = keys[i] & mask;
+      eq = km == prefix;
+      keep = km > prefix;
     }
-    // a 32-wide chunk can straddle the region boundary: rank equal keys per region
-    const uint32_t b_eq0 = __ballot_sync(0xffffffffu, eq && region == 0);
-    const uint32_t b_eq1 = __ballot_sync(0xffffffffu, eq && region == 1);
-    if (eq) {
-      const int rank = eq_seen[region] + __popc((region == 0 ? b_eq0 : b_eq1) & lt_mask);
-      keep = rank < th[region].take_equal;
+    const uint32_t b_eq = __ballot_sync(0xffffffffu, eq);
+    if (b_eq != 0u) {
+      // equal keys are taken lowest index first, counted per region (a 32-wide chunk can
+      // straddle the region boundary)
+      const uint32_t second_lanes = __ballot_sync(0xffffffffu, second);
+      const uint32_t b_eq0 = b_eq & ~second_lanes, b_eq1 = b_eq & second_lanes;
+      if (eq) {
+        const int rank = second ? eq_seen1 + __popc(b_eq1 & lt_mask) : eq_seen0 + __popc(b_eq0 & lt_mask);
+        keep = rank < (second ? th[1].take_equal : th[0].take_equal);
+      }
+      eq_seen0 += __popc(b_eq0);
+      eq_seen1 += __popc(b_eq1);
     }
-    eq_seen[0] += __popc(b_eq0);
-    eq_seen[1] += __popc(b_eq1);
     const uint32_t b_keep = __ballot_sync(0xffffffffu, keep);
     if (keep) dst[run + __popc(b_keep & lt_mask)] = i;
     run += __popc(b_keep);
