@@ -121,6 +121,30 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
                                           sparsed_pattern *out, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The switch step without a second Q K^T pass. Algorithm 1 runs full attention at the switch
+ * step and then computes A' = avgpool(A) from the same Q and K; A' can be formed from row
+ * statistics of that very full-attention pass:
+ *   sparsed_attn_full_stats   = sparsed_attn_full that also records, for every query row and
+ *                               every 64-key tile, log2 of the tile's share of the row's softmax
+ *                               denominator (tile_stats, device fp32, sparsed_tile_stats_bytes()
+ *                               bytes, layout [batch*heads_q][ceil(seq_len/64)][seq_len]);
+ *                               lse is required here.
+ *   sparsed_select_from_stats = pools those statistics into A' (2^(stat - LSE) is the
+ *                               probability mass a row puts on a tile), ranks it as
+ *                               sparsed_select_pattern does (Eq. 5 / Eq. 6) and writes the CSR
+ *                               pattern; scores_out_or_null optionally receives A'.
+ * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; seq_len <= 131072 for
+ * the selection (UNSUPPORTED beyond). Both buffers are caller-owned device memory.
+ */
+sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, size_t *out_bytes); /* host only */
+sparsed_status sparsed_attn_full_stats(const sparsed_shape *shape, const void *q, const void *k, const void *v,
+                                       void *o, float *lse, float *tile_stats, void *ws, size_t ws_bytes,
+                                       void *cuda_stream);
+sparsed_status sparsed_select_from_stats(const sparsed_shape *shape, const sparsed_select_params *params,
+                                         const float *lse, const float *tile_stats, sparsed_pattern *out,
+                                         float *scores_out_or_null, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * Block-sparse attention, O = softmax((Q K^T + M_S) / sqrt(d)) V with M_S the 0 / -inf block
  * mask given by `pattern` (Eq. 3 and Eq. 4; the "Sparse Reusing" branch of Algorithm 1).
  * Accepts any CSR whose rows are ascending and in range (not only selected ones); a query

@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_schedule_mode", "sparsed_switch_step", "sparsed_kept_per_row", "sparsed_workspace_bytes",
     "sparsed_workspace_init", "sparsed_pattern_validate", "sparsed_last_device_status",
     "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
+    "sparsed_tile_stats_bytes", "sparsed_attn_full_stats", "sparsed_select_from_stats",
 )
 
 
@@ -74,6 +75,9 @@ def load_library() -> ctypes.CDLL:
     lib.sparsed_attn_full.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_pattern.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
+    lib.sparsed_tile_stats_bytes.argtypes = [P(Shape), P(sz)]
+    lib.sparsed_attn_full_stats.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sparsed_select_from_stats.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_from_scores.argtypes = [P(SelectParams), vp, i32, i32, i32, P(Pattern), vp, sz, vp]
     lib.sparsed_attn_sparse.argtypes = [P(Shape), P(Pattern), vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_schedule_mode.argtypes = [i32, i32, f64]
@@ -200,6 +204,38 @@ def sparsed_select_pattern(q, k, params: SelectParams, pattern: Pattern, ws: tor
         lse.data_ptr() if lse is not None else None, ctypes.byref(pattern),
         scores_out.data_ptr() if scores_out is not None else None, ws.data_ptr(), ws.numel(), _stream(q)),
         "sparsed_select_pattern")
+
+
+def sparsed_tile_stats_bytes(shape: Shape) -> int:
+    out = ctypes.c_size_t()
+    _check(load_library().sparsed_tile_stats_bytes(ctypes.byref(shape), ctypes.byref(out)), "sparsed_tile_stats_bytes")
+    return int(out.value)
+
+
+def new_tile_stats(q: torch.Tensor) -> torch.Tensor:
+    """Caller-owned buffer for sparsed_attn_full_stats: fp32 [B*Hq, ceil(L/64), L]."""
+    B, Hq, L, _ = q.shape
+    return torch.empty(B * Hq, (L + 63) // 64, L, dtype=torch.float32, device=q.device)
+
+
+def sparsed_attn_full_stats(q, k, v, o, lse: torch.Tensor, tile_stats: torch.Tensor, ws: torch.Tensor,
+                            softmax_scale: float = 0.0, shape: Optional[Shape] = None) -> None:
+    shape = shape or make_shape(q, k, v, o, softmax_scale)
+    assert tile_stats.numel() * 4 >= sparsed_tile_stats_bytes(shape) and tile_stats.dtype == torch.float32
+    _check(load_library().sparsed_attn_full_stats(ctypes.byref(shape), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                                  o.data_ptr(), lse.data_ptr(), tile_stats.data_ptr(), ws.data_ptr(),
+                                                  ws.numel(), _stream(q)), "sparsed_attn_full_stats")
+
+
+def sparsed_select_from_stats(q, k, params: SelectParams, lse: torch.Tensor, tile_stats: torch.Tensor,
+                              pattern: Pattern, ws: torch.Tensor, scores_out: Optional[torch.Tensor] = None,
+                              shape: Optional[Shape] = None) -> None:
+    """q and k only provide the shape here; the kernels read lse and tile_stats."""
+    shape = shape or make_shape(q, k)
+    _check(load_library().sparsed_select_from_stats(
+        ctypes.byref(shape), ctypes.byref(params), lse.data_ptr(), tile_stats.data_ptr(), ctypes.byref(pattern),
+        scores_out.data_ptr() if scores_out is not None else None, ws.data_ptr(), ws.numel(), _stream(lse)),
+        "sparsed_select_from_stats")
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

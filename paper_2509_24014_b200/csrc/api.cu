@@ -263,8 +263,9 @@ sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stre
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
-sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
-                                 float* lse_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
+static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
+                                     float* lse_or_null, float* tile_lse_or_null, void* ws, size_t ws_bytes,
+                                     void* cuda_stream) {
   Resolved rs;
   sparsed_status st = check_shape(shape, true, &rs);
   if (st != SPARSED_OK) return st;
@@ -282,6 +283,7 @@ sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, cons
   p.o_stride_h = rs.o[1];
   p.o_stride_t = rs.o[2];
   p.lse = lse_or_null;
+  p.tile_lse = tile_lse_or_null;
   p.seq_len = shape->seq_len;
   p.heads_q = shape->heads_q;
   p.group = shape->heads_q / shape->heads_kv;
@@ -291,6 +293,59 @@ sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, cons
   p.col_idx = nullptr;
   p.status = static_cast<DeviceStatus*>(ws);
   cudaError_t e = launch_attn_dense(tq, tk, tv, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
+}
+
+sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
+                                 float* lse_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return attn_full_impl(shape, q, k, v, o, lse_or_null, nullptr, ws, ws_bytes, cuda_stream);
+}
+
+sparsed_status sparsed_tile_stats_bytes(const sparsed_shape* shape, size_t* out_bytes) {
+  if (shape == nullptr || out_bytes == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+  const size_t tiles = (static_cast<size_t>(shape->seq_len) + 63) / 64;
+  *out_bytes = static_cast<size_t>(shape->batch) * shape->heads_q * tiles * static_cast<size_t>(shape->seq_len) * 4;
+  return SPARSED_OK;
+}
+
+sparsed_status sparsed_attn_full_stats(const sparsed_shape* shape, const void* q, const void* k, const void* v,
+                                       void* o, float* lse, float* tile_stats, void* ws, size_t ws_bytes,
+                                       void* cuda_stream) {
+  if (lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
+  return attn_full_impl(shape, q, k, v, o, lse, tile_stats, ws, ws_bytes, cuda_stream);
+}
+
+sparsed_status sparsed_select_from_stats(const sparsed_shape* shape, const sparsed_select_params* params,
+                                         const float* lse, const float* tile_stats, sparsed_pattern* out,
+                                         float* scores_out_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+  if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  const int nb = shape->seq_len / params->block_size;
+  int pb = 0, k_pre = 0, k_gen = 0;
+  sparsed_status st = kept_counts(params, nb, &pb, &k_pre, &k_gen);
+  if (st != SPARSED_OK) return st;
+  if (lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (shape->seq_len > 131072) return SPARSED_ERR_UNSUPPORTED;
+  if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
+    return st;
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_arch()) != SPARSED_OK) return st;
+  PoolParams pp;
+  pp.tile_lse = tile_stats;
+  pp.lse = lse;
+  pp.scores = scores_out_or_null;
+  pp.row_ptr = out->row_ptr;
+  pp.col_idx = out->col_idx;
+  pp.seq_len = shape->seq_len;
+  pp.block_size = params->block_size;
+  pp.pb = pb;
+  pp.k_pre = k_pre;
+  pp.k_gen = k_gen;
+  pp.bh = shape->batch * shape->heads_q;
+  cudaError_t e = launch_pool_select(pp, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
@@ -320,6 +375,7 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   p.o_stride_h = rs.o[1];
   p.o_stride_t = rs.o[2];
   p.lse = nullptr;
+  p.tile_lse = nullptr;
   p.seq_len = shape->seq_len;
   p.heads_q = shape->heads_q;
   p.group = shape->heads_q / shape->heads_kv;

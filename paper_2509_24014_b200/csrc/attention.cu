@@ -356,6 +356,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       }
       l += sum;
+      if (p.tile_lse != nullptr) {
+        // switch step: keep log2 of this tile's share of the row's softmax denominator, from
+        // which the pooled block scores are formed later without a second Q K^T pass
+        const int row_g = q_row0 + tid;
+        if (tid < kRowsQ && row_g < p.seq_len)
+          p.tile_lse[(static_cast<int64_t>(bh) * num_tiles + t) * p.seq_len + row_g] = m_used + __log2f(sum);
+      }
       TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();

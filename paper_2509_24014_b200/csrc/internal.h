@@ -14,6 +14,7 @@ struct AttnParams {
   void* o;                 // bf16 [B,Hq,L,D]
   int64_t o_stride_b, o_stride_h, o_stride_t;
   float* lse;              // fp32 [B,Hq,L] or null
+  float* tile_lse;         // fp32 [B*Hq, ceil(L/64), L] or null: base-2 log-sum-exp of each row over each 64-key tile
   int seq_len;
   int heads_q;
   int group;               // heads_q / heads_kv
@@ -43,6 +44,19 @@ struct ScoreParams {
 // Largest number of key blocks per row the pooled-scoring kernel can rank in its own tail.
 constexpr int kFusedTopkMaxBlocks = 1024;
 
+// Parameters of the kernel that pools per-tile row statistics into A' and ranks it.
+struct PoolParams {
+  const float* tile_lse;   // fp32 [B*Hq, tiles, L], base-2
+  const float* lse;        // fp32 [B,Hq,L], natural log
+  float* scores;           // fp32 [B,Hq,nb,nb] or null
+  int32_t* row_ptr;
+  int32_t* col_idx;
+  int seq_len;
+  int block_size;          // 64 or 128
+  int pb, k_pre, k_gen;
+  int bh;                  // B * Hq
+};
+
 struct TopkParams {
   const float* scores;     // fp32 [rows, nb]
   int32_t* row_ptr;
@@ -62,6 +76,7 @@ cudaError_t launch_row_stats(const CUtensorMap& tq, const CUtensorMap& tk, const
 cudaError_t launch_pooled_scores(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int batch,
                                  cudaStream_t stream);
 cudaError_t launch_topk_csr(const TopkParams& p, cudaStream_t stream);
+cudaError_t launch_pool_select(const PoolParams& p, cudaStream_t stream);
 cudaError_t launch_pattern_validate(const int32_t* row_ptr, const int32_t* col_idx, int rows, int nb,
                                     int64_t capacity, int* bad_flag, cudaStream_t stream);
 

@@ -1,0 +1,148 @@
+// Pattern selection from the row statistics of the switch step's full-attention pass
+// ("Isolated Selection": A' = avgpool(A, block_size), then Eq. 5 / Eq. 6), without a second
+// Q K^T pass.
+//
+// The dense attention kernel can record, for every query row i and every 64-key tile t,
+// v[t][i] = log2 sum_{j in t} 2^(s_ij), the tile's share of the row's softmax denominator.
+// With the row's final log-sum-exp, 2^(v[t][i] - LSE_i) is exactly the probability mass row i
+// puts on tile t, so A'[ib][jb] is the sum of that mass over the rows of block ib and the tiles
+// of block jb, divided by block_size^2.
+//
+// One CTA owns one 128-row query tile of one (batch, head): thread r owns row r. Statistics
+// are read coalesced (row-fastest layout), exponentiated, transposed through padded shared
+// memory in chunks of 128 tiles, and summed per tile in a fixed order (bitwise reproducible).
+// The CTA then holds its block-row(s) of A' in shared memory, optionally writes them out, and
+// warp 0 ranks them (warp_select_row) and writes the CSR lists. HBM-bound:
+// 4 * L * ceil(L/64) bytes read per (batch, head).
+#include "internal.h"
+#include "topk_device.cuh"
+
+namespace sparsed {
+namespace {
+
+constexpr int kRows = 128;
+constexpr int kChunk = 64;          // tiles per transposition chunk
+constexpr int kInFlight = 16;       // loads each thread keeps in flight
+constexpr int kMaxTiles = 2048;     // seq_len <= 131072
+
+// Shared memory (dynamic, sized for the actual sequence): the transposition chunk, the per-tile
+// mass of rows 0-63 / 64-127, the ordered keys of this CTA's block-row(s), the top-k histogram.
+struct PoolSmem {
+  float (*chunk)[kRows + 1];        // [tile in chunk][row], padded against bank conflicts
+  float* tile_sum[2];               // [row half][tile]
+  uint32_t* keys[2];
+  int* hist;
+};
+
+__host__ __device__ inline size_t pool_smem_bytes(int n_tiles, int nb) {
+  return sizeof(float) * kChunk * (kRows + 1) + sizeof(float) * 2 * n_tiles + sizeof(uint32_t) * 2 * nb +
+         sizeof(int) * 256;
+}
+
+__global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams p) {
+  extern __shared__ __align__(16) uint8_t pool_smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int L = p.seq_len;
+  const int n_tiles = (L + 63) / 64;
+  PoolSmem sm;
+  {
+    float* f = reinterpret_cast<float*>(pool_smem_raw);
+    sm.chunk = reinterpret_cast<float (*)[kRows + 1]>(f);
+    f += kChunk * (kRows + 1);
+    sm.tile_sum[0] = f;
+    sm.tile_sum[1] = f + n_tiles;
+    f += 2 * n_tiles;
+    const int nb_ = L / p.block_size;
+    sm.keys[0] = reinterpret_cast<uint32_t*>(f);
+    sm.keys[1] = sm.keys[0] + nb_;
+    sm.hist = reinterpret_cast<int*>(sm.keys[1] + nb_);
+  }
+  const int num_q_tiles = (L + kRows - 1) / kRows;
+  const int q_tile = blockIdx.x % num_q_tiles;
+  const int bh = blockIdx.x / num_q_tiles;
+  const int row = q_tile * kRows + tid;
+  const bool row_valid = row < L;
+  const float lse2 = row_valid ? p.lse[static_cast<int64_t>(bh) * L + row] * 1.44269504088896341f : INFINITY;
+  const float* src = p.tile_lse + static_cast<int64_t>(bh) * n_tiles * L + row;
+
+  for (int c0 = 0; c0 < n_tiles; c0 += kChunk) {
+    const int n_here = min(kChunk, n_tiles - c0);
+    // coalesced over rows; kInFlight loads in flight per thread
+    for (int tt = 0; tt < n_here; tt += kInFlight) {
+      float v[kInFlight];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u)
+        v[u] = (row_valid && tt + u < n_here) ? __ldg(src + static_cast<int64_t>(c0 + tt + u) * L) : -INFINITY;
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u)
+        if (tt + u < n_here) sm.chunk[tt + u][tid] = fast_exp2(v[u] - lse2);
+    }
+    __syncthreads();
+    if (tid < n_here) {
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+      for (int r = 0; r < 64; ++r) s0 += sm.chunk[tid][r];
+#pragma unroll 8
+      for (int r = 64; r < 128; ++r) s1 += sm.chunk[tid][r];
+      sm.tile_sum[0][c0 + tid] = s0;
+      sm.tile_sum[1][c0 + tid] = s1;
+    }
+    __syncthreads();
+  }
+
+  const int bs = p.block_size;
+  const int nb = L / bs;
+  const float inv_area = 1.f / (static_cast<float>(bs) * static_cast<float>(bs));
+  const int rows_here = bs == 64 ? 2 : 1;
+  for (int jb = tid; jb < nb; jb += kRows) {
+    if (bs == 128) {
+      const float total = (sm.tile_sum[0][2 * jb] + sm.tile_sum[1][2 * jb]) +
+                          (sm.tile_sum[0][2 * jb + 1] + sm.tile_sum[1][2 * jb + 1]);
+      const float score = total * inv_area;
+      sm.keys[0][jb] = ordered_key(score);
+      if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + q_tile) * nb + jb] = score;
+    } else {
+#pragma unroll
+      for (int rh = 0; rh < 2; ++rh) {
+        const int ib = q_tile * 2 + rh;
+        if (ib < nb) {
+          const float score = sm.tile_sum[rh][jb] * inv_area;
+          sm.keys[rh][jb] = ordered_key(score);
+          if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + ib) * nb + jb] = score;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int k_total = p.k_pre + p.k_gen;
+    for (int rh = 0; rh < rows_here; ++rh) {
+      const int ib = bs == 64 ? q_tile * 2 + rh : q_tile;
+      if (ib >= nb) break;
+      const int64_t r = static_cast<int64_t>(bh) * nb + ib;
+      warp_select_row(sm.keys[rh], nb, p.pb, p.k_pre, p.k_gen, sm.hist, p.col_idx + r * k_total, lane);
+      if (lane == 0) {
+        p.row_ptr[r] = static_cast<int32_t>(r * k_total);
+        if (r == static_cast<int64_t>(p.bh) * nb - 1) p.row_ptr[r + 1] = static_cast<int32_t>((r + 1) * k_total);
+      }
+      __syncwarp();
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_pool_select(const PoolParams& p, cudaStream_t stream) {
+  const int n_tiles = (p.seq_len + 63) / 64;
+  if (n_tiles > kMaxTiles) return cudaErrorInvalidValue;
+  const int smem = static_cast<int>(pool_smem_bytes(n_tiles, p.seq_len / p.block_size));
+  cudaError_t e = cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  const int num_q_tiles = (p.seq_len + kRows - 1) / kRows;
+  const long long ctas = static_cast<long long>(p.bh) * num_q_tiles;
+  if (ctas <= 0) return cudaSuccess;
+  pool_select_kernel<<<static_cast<unsigned>(ctas), kRows, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace sparsed
