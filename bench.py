@@ -2,8 +2,9 @@
 """Benchmark of the SparseD attention hot path on B200.
 
 One "step" is one pass of the whole hot path over one synthetic batch of the 64k workload:
-schedule helper -> dense attention (+LSE) -> pattern selection (pooled scoring, top-k, CSR)
--> block-sparse attention on the selected pattern. The headline value is the block-sparse
+schedule helper -> dense attention that also records per-tile row statistics -> pattern
+selection from those statistics (pooling to A', isolated top-k, CSR) -> block-sparse attention
+on the selected pattern. The headline value is the block-sparse
 attention throughput in TFLOP/s counted on kept-block FLOPs (4 * bs^2 * D * nnz), with its
 fraction of the measured bf16 peak and the wall-time speedup over the library's own dense
 kernel reported beside it.
@@ -233,6 +234,7 @@ def run_ours(args, cfg):
     shape_qkvo = sd.make_shape(q, k, v, o_full)
     shape_qk = sd.make_shape(q, k)
     ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_PATTERN, shape_qk, params), dev)
+    tile_stats = sd.new_tile_stats(q)
     total_steps, skip = max(cfg.total_steps, 2), (cfg.skip if cfg.total_steps > 1 else 0.5)
     s_switch = sd.sparsed_switch_step(total_steps, skip)
 
@@ -247,9 +249,9 @@ def run_ours(args, cfg):
                 e = ev(); e.record(); marks.append(e)
         mark()
         assert sd.sparsed_schedule_mode(s_switch, total_steps, skip) == sd.MODE_FULL_AND_SELECT
-        sd.sparsed_attn_full(q, k, v, o_full, lse, ws, shape=shape_qkvo)
+        sd.sparsed_attn_full_stats(q, k, v, o_full, lse, tile_stats, ws, shape=shape_qkvo)
         mark()
-        sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse, shape=shape_qk)
+        sd.sparsed_select_from_stats(q, k, params, lse, tile_stats, pat, ws, shape=shape_qk)
         mark()
         assert sd.sparsed_schedule_mode(s_switch + 1, total_steps, skip) == sd.MODE_SPARSE
         sd.sparsed_attn_sparse(q, k, v, o_sparse, pat, ws, shape=shape_qkvo)
@@ -372,15 +374,36 @@ def run_ours(args, cfg):
                 "traffic": NCU_DRAM_TRAFFIC.get(("topk_csr_kernel", cfg.name)),
                 "note": "event time of a single launch includes launch latency; L2 flushed before it"}
 
+    def two_pass_select():
+        """The alternative selection path (a second Q K^T pass: pooled scoring with its fused
+        top-k), timed outside the step for comparison; a dense contraction of 2*L^2*D per head."""
+        times = []
+        for _ in range(3):
+            a, b = ev(), ev()
+            a.record()
+            sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse, shape=shape_qk)
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        r = tensor_roofline("score_kernel (two-pass selection, not in the step)", dense_flops(cfg) / 2, times[1:])
+        return r
+
     roof_dense = tensor_roofline("attn_kernel<dense>", dense_flops(cfg), full_ms)
     roof_sparse = tensor_roofline("attn_kernel<sparse>", sparse_flops(cfg, nnz), sparse_ms)
     # selection = pooled-scoring kernel (a dense QK^T contraction, 2*L^2*D per head) + top-k/CSR kernel
-    fused_topk = nb <= 1024   # the scoring kernel ranks its own block-rows up to 1024 blocks per row
-    launches_per_step = 3 if fused_topk else 4
-    roof_select = tensor_roofline("score_kernel", dense_flops(cfg) / 2, select_ms)
+    launches_per_step = 3
+    # selection from the recorded statistics is HBM-bound: it reads 4*L*ceil(L/64) bytes per head
+    stats_bytes = tile_stats.numel() * 4 + lse.numel() * 4 + 4 * nnz + 4 * (B * Hq * nb + 1)
+    sel_ms = sum(select_ms) / len(select_ms)
+    sel_gbs = stats_bytes / (sel_ms * 1e-3) / 1e9
+    roof_select = {"kernel": "pool_select_kernel", "bound": "hbm", "achieved": sel_gbs, "peak": peaks["hbm_gbs"],
+                   "unit": "GB/s", "frac": sel_gbs / peaks["hbm_gbs"], "peak_source": f"HBM copy, {tag}",
+                   "avg_launch_ms": sel_ms, "algorithmic_bytes": stats_bytes,
+                   "traffic": NCU_DRAM_TRAFFIC.get(("pool_select_kernel", cfg.name))}
     roof_topk = topk_roofline()
+    roof_two_pass = two_pass_select()
     dominant = max((roof_dense, roof_select, roof_sparse), key=lambda r: r["avg_launch_ms"])
-    roof_all = [roof_dense, roof_select, roof_topk, roof_sparse]
+    roof_all = [roof_dense, roof_select, roof_sparse, roof_two_pass, roof_topk]
 
     # ---- CPU oracle beside it (bounded sample of the same workload) ----------------------
     cpu = None
@@ -398,7 +421,7 @@ def run_ours(args, cfg):
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": n, "warmup": args.warmup,
         "ms_per_step": total_ms / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "step": "attn_full+lse -> select_pattern -> attn_sparse",
+        "config": {"workload": workload_name(cfg), "step": "attn_full_stats -> select_from_stats -> attn_sparse",
                    "kept_per_row": [k_pre, k_gen], "nnz": nnz, "density": nnz / (B * Hq * nb * nb),
                    "l2": "inputs larger than L2 (Q,K,V,O = %.2f GB per pass)" % (4 * q.numel() * 2 / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
@@ -407,15 +430,16 @@ def run_ours(args, cfg):
         "pct_bf16_nominal_2250": 100.0 * per_gpu_sparse / 2250.0,
         "dense_tflops": dense_tflops,
         "speedup_vs_dense": full_total / sparse_total, "ideal_speedup": nb / (k_pre + k_gen),
-        "phase_ms": {"attn_full": full_total / n, "select_pattern": select_total / n, "attn_sparse": sparse_total / n},
+        "phase_ms": {"attn_full_stats": full_total / n, "select_from_stats": select_total / n,
+                     "attn_sparse": sparse_total / n},
         "roofline": dominant, "roofline_by_kernel": roof_all,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "pinned host Q,K,V -> device, sparsed_attn_sparse, O -> pinned host", "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": launches_per_step * n,
-        "launches_per_step": {"attn_kernel<dense>": 1, "score_kernel (pooled scoring + fused top-k/CSR)": 1,
-                              "topk_csr_kernel": 0 if fused_topk else 1, "attn_kernel<sparse>": 1},
+        "launches_per_step": {"attn_kernel<dense> (+ tile statistics)": 1,
+                              "pool_select_kernel (pooling + top-k + CSR)": 1, "attn_kernel<sparse>": 1},
         "clocks": clocks, "peaks": peaks,
     }
     print(json.dumps(line))
@@ -453,6 +477,138 @@ def run_topk_only(args, cfg):
                       "frac_of_hbm_peak": nbytes / ms / 1e6 / peaks["hbm_gbs"], "l2": "flushed before each launch"}))
 
 
+def _ev():
+    return torch.cuda.Event(enable_timing=True)
+
+
+def run_schedule_loop(args, cfg):
+    """The denoising-loop workloads: every step asks the schedule helper for its mode and makes the
+    matching library call(s). c4: one layer, 64 steps, fresh noise on Q/K/V each step, pattern selected
+    once at the switch step and reused. c5: four layers, 256 steps, the same Q/K/V every step.
+    Reports per-phase times, the speedup over all-full attention and (c4) the final-step output error
+    against the oracle on sampled rows. Only library calls are inside the timed events; drawing the
+    inputs is not."""
+    import paper_2509_24014_b200 as sd
+    from oracle import sparsed_oracle as orc
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    T, skip, bs = cfg.total_steps, cfg.skip, cfg.block_size
+    s_switch = sd.sparsed_switch_step(T, skip)
+    B, Hq, L, nb = cfg.batch, cfg.heads_q, cfg.seq_len, cfg.num_blocks
+    params = sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)
+    k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
+    ws = sd.new_workspace(256, dev)
+    layers = []
+    for layer in range(cfg.layers):
+        base = syn.make_base(cfg, dev, layer) if cfg.step_noise > 0 else None
+        qkv = None if base is not None else syn.make_qkv(cfg, dev, layer)
+        pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+        layers.append({"base": base, "qkv": qkv, "pat": pat, "row_ptr": row_ptr, "col_idx": col_idx})
+    o = torch.empty(B, Hq, L, cfg.head_dim, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+    stats = torch.empty(B * Hq, (L + 63) // 64, L, dtype=torch.float32, device=dev)
+    times = {"full": [], "select": [], "sparse": []}
+    sample_heads = [0, Hq // 2, Hq - 1]
+    sample_blocks = [0, nb // 2 + 1, nb - 1]
+    switch_qk = {}
+    final = {}
+    # warm-up of the three kernels
+    q, k, v = layers[0]["qkv"] if layers[0]["qkv"] is not None else syn.make_qkv(cfg, dev, 0, step=0, base=layers[0]["base"])
+    for _ in range(2):
+        sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+        sd.sparsed_select_from_stats(q, k, params, lse, stats, layers[0]["pat"], ws)
+        sd.sparsed_attn_sparse(q, k, v, o, layers[0]["pat"], ws)
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    for t in range(1, T + 1):
+        mode = sd.sparsed_schedule_mode(t, T, skip)
+        for li, lay in enumerate(layers):
+            if lay["base"] is not None:
+                q, k, v = syn.make_qkv(cfg, dev, li, step=t, base=lay["base"])
+            else:
+                q, k, v = lay["qkv"]
+            a, b, c = _ev(), _ev(), _ev()
+            a.record()
+            if mode == sd.MODE_FULL:
+                sd.sparsed_attn_full(q, k, v, o, None, ws)
+                b.record()
+                times["full"].append((a, b))
+            elif mode == sd.MODE_FULL_AND_SELECT:
+                sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+                b.record()
+                sd.sparsed_select_from_stats(q, k, params, lse, stats, lay["pat"], ws)
+                c.record()
+                times["full"].append((a, b))
+                times["select"].append((b, c))
+                if cfg.step_noise > 0:
+                    for h in sample_heads:
+                        switch_qk[h] = (q[0, h].to("cpu"), k[0, h // (Hq // cfg.heads_kv)].to("cpu"))
+            else:
+                sd.sparsed_attn_sparse(q, k, v, o, lay["pat"], ws)
+                b.record()
+                times["sparse"].append((a, b))
+            if t == T and li == 0 and cfg.step_noise > 0:
+                torch.cuda.synchronize()
+                for h in sample_heads:
+                    hk = h // (Hq // cfg.heads_kv)
+                    final[h] = (q[0, h].to("cpu"), k[0, hk].to("cpu"), v[0, hk].to("cpu"), o[0, h].to("cpu"))
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    code, where = sd.sparsed_last_device_status(ws)
+    if code != 0:
+        raise RuntimeError(f"device status {code} at {where}")
+    ms = {kk: [x.elapsed_time(y) for x, y in vv] for kk, vv in times.items()}
+    med = {kk: (statistics.median(vv) if vv else None) for kk, vv in ms.items()}
+    total = sum(sum(vv) for vv in ms.values())
+    n_calls = cfg.layers * T
+    out = {"workload": workload_name(cfg) + f", T={T}, skip={skip}, layers={cfg.layers}", "switch_step": s_switch,
+           "calls": {kk: len(vv) for kk, vv in ms.items()}, "median_ms": med,
+           "total_attention_ms": total, "speedup_sparse_vs_full_step": med["full"] / med["sparse"],
+           "ideal_step_speedup": nb / (k_pre + k_gen), "kept_per_row": [k_pre, k_gen],
+           "dense_tflops_median": dense_flops(cfg) / med["full"] / 1e9,
+           "sparse_tflops_median": sparse_flops(cfg, int(layers[0]["pat"].nnz)) / med["sparse"] / 1e9,
+           "wall_s_including_input_generation": wall}
+    if args.all_full:
+        # the same number of calls with full attention only, timed as one loop
+        q, k, v = layers[0]["qkv"] if layers[0]["qkv"] is not None else syn.make_qkv(cfg, dev, 0, step=1, base=layers[0]["base"])
+        a, b = _ev(), _ev()
+        a.record()
+        for _ in range(n_calls):
+            sd.sparsed_attn_full(q, k, v, o, None, ws)
+        b.record()
+        torch.cuda.synchronize()
+        out["all_full_attention_ms"] = a.elapsed_time(b)
+        out["speedup_whole_schedule_measured"] = out["all_full_attention_ms"] / total
+    else:
+        out["all_full_attention_ms_estimated"] = n_calls * med["full"]
+        out["speedup_whole_schedule_estimated"] = n_calls * med["full"] / total
+    n_full = len(ms["full"])
+    out["ideal_whole_schedule_speedup"] = n_calls / (n_full + (n_calls - n_full) * (k_pre + k_gen) / nb)
+    if final:
+        # final-step output error on sampled rows: the oracle attends on the final step's tensors with
+        # (a) the GPU's pattern and (b) its own fp64 selection from the switch step's tensors
+        f64 = lambda x: x.to(torch.float64).numpy()
+        rp, ci = layers[0]["row_ptr"].cpu().numpy(), layers[0]["col_idx"].cpu().numpy()
+        pb = cfg.prefill_len // bs
+        err_gpu_pat, err_own_pat, same_lists = [], [], []
+        for h in sample_heads:
+            qh, kh, vh, oh = (f64(x) for x in final[h])
+            qs, ks = (f64(x) for x in switch_qk[h])
+            for ib in sample_blocks:
+                r = h * nb + ib
+                gpu_list = list(ci[rp[r]:rp[r + 1]])
+                own_list = orc.select_row(orc.head_pooled_row(qs, ks, ib, bs), pb, cfg.keep_ratio)
+                rows = slice(ib * bs, (ib + 1) * bs)
+                err_gpu_pat.append(np.abs(oh[rows] - orc.head_sparse_rows(qh, kh, vh, ib, gpu_list, bs)).max())
+                err_own_pat.append(np.abs(oh[rows] - orc.head_sparse_rows(qh, kh, vh, ib, own_list, bs)).max())
+                same_lists.append(gpu_list == own_list)
+        out["final_step_max_abs_err_vs_oracle_same_pattern"] = float(max(err_gpu_pat))
+        out["final_step_max_abs_err_vs_oracle_own_pattern"] = float(max(err_own_pat))
+        out["sampled_rows"] = len(same_lists)
+        out["sampled_rows_with_identical_lists"] = int(sum(same_lists))
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -464,9 +620,14 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=4, help="row blocks per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only-topk", action="store_true", help="run only the stand-alone ranking kernel")
+    ap.add_argument("--schedule-loop", action="store_true",
+                    help="run the config's whole denoising schedule (c4: 64 steps, c5: 4 layers x 256 steps)")
+    ap.add_argument("--all-full", action="store_true", help="with --schedule-loop: also time all-full attention")
     args = ap.parse_args()
     cfg = syn.CONFIGS[args.config]
-    if args.only_topk:
+    if args.schedule_loop:
+        run_schedule_loop(args, cfg)
+    elif args.only_topk:
         run_topk_only(args, cfg)
     elif args.impl == "reference":
         run_reference(args, cfg)

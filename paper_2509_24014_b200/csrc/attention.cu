@@ -72,7 +72,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
-  const int lane = tid & 31;
   constexpr int kTilesPerBlock = kBlock / kTileN;
 
   // ---- work item -----------------------------------------------------------------------
