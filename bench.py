@@ -32,6 +32,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2509_24014_b200 import replicas  # noqa: E402
 from paper_2509_24014_b200 import synthetic as syn  # noqa: E402
 
 METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at 64k"
@@ -231,7 +232,7 @@ def run_ours(args, cfg):
     sd.load_library()
     peaks = load_peaks()
 
-    cfg_r = cfg.with_(seed=cfg.seed + 1000 * rank)
+    cfg_r = cfg.with_(seed=replicas.replica_seed(cfg.seed, rank))
     q, k, v = syn.make_qkv(cfg_r, dev)
     B, Hq, L, D = q.shape
     nb = cfg.num_blocks
@@ -301,12 +302,8 @@ def run_ours(args, cfg):
     nnz = int(pat.nnz)
 
     # max over ranks of the timed quantities
-    if dist is not None:
-        t = torch.tensor([total_ms, sparse_total, sum(full_ms), sum(select_ms)], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, sparse_total, full_total, select_total = t.tolist()
-    else:
-        full_total, select_total = sum(full_ms), sum(select_ms)
+    total_ms, sparse_total, full_total, select_total = replicas.max_over_ranks(
+        [total_ms, sparse_total, sum(full_ms), sum(select_ms)], dist, dev)
 
     n = args.steps
     value = world * n * sparse_flops(cfg, nnz) / (sparse_total * 1e-3) / 1e12
@@ -336,10 +333,7 @@ def run_ours(args, cfg):
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = t.item()
+    e2e_ms = replicas.max_over_ranks([e2e_ms], dist, dev)[0]
     e2e_value = world * e2e_steps * sparse_flops(cfg, nnz) / (e2e_ms * 1e-3) / 1e12
 
     if rank != 0:

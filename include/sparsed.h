@@ -180,6 +180,18 @@ sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape *shape,
 sparsed_status sparsed_workspace_init(void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Fixed comparison patterns in the same CSR form (the sliding-window and sink-plus-window
+ * baselines of the paper's "Experimental Setting", expressed in blocks): query block i keeps the
+ * key blocks [0, sink_blocks) and those with |j - i| <= (window_blocks - 1) / 2 (a symmetric
+ * window, since the attention is bidirectional). Lists are ascending; rows near the edges are
+ * shorter. `out`: row_ptr/col_idx/col_capacity are inputs (capacity is checked against the exact
+ * count, returned in nnz). Device arrays are written asynchronously on the stream.
+ */
+sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int32_t num_blocks, int32_t block_size,
+                                            int32_t sink_blocks, int32_t window_blocks, sparsed_pattern *out,
+                                            void *cuda_stream);
+
+/*
  * Checks a pattern on the device: row_ptr monotone and within capacity, every list strictly
  * ascending and within [0, num_blocks), no empty row. Synchronises the stream. Returns
  * SPARSED_OK or SPARSED_ERR_PATTERN. (No paper counterpart: a guard for user-built masks.)

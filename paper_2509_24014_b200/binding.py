@@ -24,6 +24,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_workspace_init", "sparsed_pattern_validate", "sparsed_last_device_status",
     "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
     "sparsed_tile_stats_bytes", "sparsed_attn_full_stats", "sparsed_select_from_stats",
+    "sparsed_build_window_pattern",
 )
 
 
@@ -75,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.sparsed_attn_full.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_pattern.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
+    lib.sparsed_build_window_pattern.argtypes = [i32, i32, i32, i32, i32, i32, P(Pattern), vp]
     lib.sparsed_tile_stats_bytes.argtypes = [P(Shape), P(sz)]
     lib.sparsed_attn_full_stats.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_from_stats.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
@@ -269,6 +271,20 @@ def sparsed_attn_sparse(q, k, v, o, pattern: Pattern, ws: torch.Tensor, softmax_
     _check(load_library().sparsed_attn_sparse(ctypes.byref(shape), ctypes.byref(pattern), q.data_ptr(),
                                               k.data_ptr(), v.data_ptr(), o.data_ptr(), ws.data_ptr(), ws.numel(),
                                               _stream(q)), "sparsed_attn_sparse")
+
+
+def sparsed_build_window_pattern(batch: int, heads_q: int, num_blocks: int, block_size: int, sink_blocks: int,
+                                 window_blocks: int, device):
+    """Sliding-window (+ sink) comparison pattern as CSR; returns (Pattern, row_ptr, col_idx)."""
+    half = (window_blocks - 1) // 2
+    cap = batch * heads_q * num_blocks * min(num_blocks, 2 * half + 1 + max(sink_blocks, 0))
+    row_ptr = torch.zeros(batch * heads_q * num_blocks + 1, dtype=torch.int32, device=device)
+    col_idx = torch.zeros(max(cap, 1), dtype=torch.int32, device=device)
+    pat = Pattern(row_ptr.data_ptr(), col_idx.data_ptr(), col_idx.numel(), 0, 0, 0, 0, 0)
+    _check(load_library().sparsed_build_window_pattern(batch, heads_q, num_blocks, block_size, sink_blocks,
+                                                       window_blocks, ctypes.byref(pat), _stream(row_ptr)),
+           "sparsed_build_window_pattern")
+    return pat, row_ptr, col_idx
 
 
 def sparsed_pattern_validate(pattern: Pattern, ws: torch.Tensor) -> bool:

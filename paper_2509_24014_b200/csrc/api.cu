@@ -463,6 +463,31 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   return run_topk(scores, shape->batch, shape->heads_q, nb, params->block_size, pb, k_pre, k_gen, out, stream);
 }
 
+sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int32_t num_blocks, int32_t block_size,
+                                            int32_t sink_blocks, int32_t window_blocks, sparsed_pattern* out,
+                                            void* cuda_stream) {
+  if (batch < 1 || heads_q < 1 || num_blocks < 1 || sink_blocks < 0 || window_blocks < 1) return SPARSED_ERR_INVALID_ARG;
+  if (block_size != 64 && block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (num_blocks > 16384) return SPARSED_ERR_UNSUPPORTED;
+  if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  const int sink = sink_blocks < num_blocks ? sink_blocks : num_blocks;
+  const int half = (window_blocks - 1) / 2;
+  const int64_t per_head = window_pattern_nnz_per_head(num_blocks, sink, half);
+  const int64_t bh = static_cast<int64_t>(batch) * heads_q;
+  const int64_t nnz = per_head * bh;
+  if (nnz >= INT32_MAX || bh * num_blocks >= INT32_MAX) return SPARSED_ERR_UNSUPPORTED;
+  if (out->col_capacity < nnz) return SPARSED_ERR_PATTERN;
+  cudaError_t e = launch_window_pattern(out->row_ptr, out->col_idx, static_cast<int>(bh), num_blocks, sink, half,
+                                        static_cast<int>(per_head), static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return cuda_fail(e);
+  out->nnz = nnz;
+  out->block_size = block_size;
+  out->num_blocks = num_blocks;
+  out->batch = batch;
+  out->heads_q = heads_q;
+  return SPARSED_OK;
+}
+
 sparsed_status sparsed_pattern_validate(const sparsed_pattern* pattern, void* ws, size_t ws_bytes, void* cuda_stream) {
   if (pattern == nullptr || pattern->row_ptr == nullptr || pattern->col_idx == nullptr) return SPARSED_ERR_PATTERN;
   if (pattern->batch < 1 || pattern->heads_q < 1 || pattern->num_blocks < 1) return SPARSED_ERR_PATTERN;
