@@ -623,6 +623,78 @@ def run_schedule_loop(args, cfg, emit=True):
     return out
 
 
+def run_sweep(args, cfg):
+    """Timed variants of the method on one workload shape (the paper's ablation axes, latency only):
+    keep ratio, isolated vs plain selection, re-selecting every step, no full-attention prefix, and
+    the sliding-window / sink+window comparison patterns through the same sparse kernel."""
+    import paper_2509_24014_b200 as sd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    q, k, v = syn.make_qkv(cfg, dev)
+    B, Hq, L, D = q.shape
+    bs, nb = cfg.block_size, cfg.num_blocks
+    o = torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+    stats = sd.new_tile_stats(q)
+    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_PATTERN, sd.make_shape(q, k),
+                                                      sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)), dev)
+
+    def timed(fn, reps=5):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = _ev(), _ev()
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+
+    full_ms = timed(lambda: sd.sparsed_attn_full(q, k, v, o, None, ws), reps=3)
+    full_stats_ms = timed(lambda: sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws), reps=3)
+    rows = []
+    for rho in (0.05, 0.1, 0.2, 0.3, 0.5):
+        for p_len in sorted({0, cfg.prefill_len, L // 2}):
+            params = sd.make_params(bs, rho, p_len)
+            k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
+            pat, rp, ci = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+            sel_ms = timed(lambda: sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws))
+            sp_ms = timed(lambda: sd.sparsed_attn_sparse(q, k, v, o, pat, ws))
+            rows.append({"keep_ratio": rho, "prefill_len": p_len, "kept_per_row": [k_pre, k_gen],
+                         "select_from_stats_ms": sel_ms, "sparse_ms": sp_ms,
+                         "sparse_tflops": sparse_flops(cfg, int(pat.nnz)) / sp_ms / 1e9,
+                         "speedup_vs_full": full_ms / sp_ms, "ideal": nb / (k_pre + k_gen)})
+    # the paper's ablation rows as per-step attention time at this shape
+    params = sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)
+    k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
+    pat, rp, ci = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+    sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws)
+    sp_ms = timed(lambda: sd.sparsed_attn_sparse(q, k, v, o, pat, ws))
+    resel_ms = timed(lambda: sd.sparsed_select_pattern(q, k, params, pat, ws, lse=None), reps=3)
+    T, skip = max(cfg.total_steps, 2), cfg.skip if cfg.total_steps > 1 else 0.2
+    s_sw = sd.sparsed_switch_step(T, skip)
+    sel_ms = timed(lambda: sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws))
+    total_sparsed = (s_sw - 1) * full_ms + full_stats_ms + sel_ms + (T - s_sw) * sp_ms
+    ablation = {
+        "T": T, "skip": skip, "switch_step": s_sw, "full_step_ms": full_ms, "sparse_step_ms": sp_ms,
+        "all_full_ms": T * full_ms, "sparsed_ms": total_sparsed,
+        "no_skipping_ms (skip=0: select at step 1)": full_stats_ms + sel_ms + (T - 1) * sp_ms,
+        "no_reuse_ms (re-select every sparse step, own QK^T pass incl. row statistics)":
+            (s_sw - 1) * full_ms + full_stats_ms + sel_ms + (T - s_sw) * (resel_ms + sp_ms),
+        "reselect_ms": resel_ms,
+    }
+    # comparison patterns: sliding window ws = l/2 and sink (10 % of the keys) + window
+    base = {}
+    for name, sink, window in (("sliding_window_ws_l/2", 0, nb // 2 + 1), ("sink10%+window_ws_l/2", max(1, nb // 10), nb // 2 + 1)):
+        wpat, wrp, wci = sd.sparsed_build_window_pattern(B, Hq, nb, bs, sink, window, dev)
+        w_ms = timed(lambda: sd.sparsed_attn_sparse(q, k, v, o, wpat, ws))
+        base[name] = {"nnz": int(wpat.nnz), "density": int(wpat.nnz) / (B * Hq * nb * nb), "sparse_ms": w_ms,
+                      "sparse_tflops": sparse_flops(cfg, int(wpat.nnz)) / w_ms / 1e9, "speedup_vs_full": full_ms / w_ms}
+    print(json.dumps({"workload": workload_name(cfg), "full_ms": full_ms, "full_with_stats_ms": full_stats_ms,
+                      "dense_tflops": dense_flops(cfg) / full_ms / 1e9, "keep_ratio_sweep": rows,
+                      "ablation_schedule_ms": ablation, "comparison_patterns": base}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -638,9 +710,12 @@ def main():
                     help="run the config's whole denoising schedule (c4: 64 steps, c5: 4 layers x 256 steps)")
     ap.add_argument("--all-full", action="store_true", help="with --schedule-loop: also time all-full attention")
     ap.add_argument("--no-schedule-loop", action="store_true", help="skip the schedule-loop summary of the default run")
+    ap.add_argument("--sweep", action="store_true", help="keep-ratio / isolation / ablation / comparison-pattern timings")
     args = ap.parse_args()
     cfg = syn.CONFIGS[args.config]
-    if args.schedule_loop:
+    if args.sweep:
+        run_sweep(args, cfg)
+    elif args.schedule_loop:
         run_schedule_loop(args, cfg)
     elif args.only_topk:
         run_topk_only(args, cfg)
