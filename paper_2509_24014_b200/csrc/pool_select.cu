@@ -22,7 +22,10 @@ namespace {
 
 constexpr int kRows = 128;
 constexpr int kChunk = 64;          // tiles per transposition chunk
-constexpr int kInFlight = 16;       // loads each thread keeps in flight
+#ifndef SPARSED_POOL_IN_FLIGHT
+#define SPARSED_POOL_IN_FLIGHT 16
+#endif
+constexpr int kInFlight = SPARSED_POOL_IN_FLIGHT;  // loads each thread keeps in flight
 constexpr int kMaxTiles = 2048;     // seq_len <= 131072
 
 // Shared memory (dynamic, sized for the actual sequence): the transposition chunk, the per-tile
