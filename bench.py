@@ -703,7 +703,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c4", choices=sorted(syn.CONFIGS))
     ap.add_argument("--cpu-rows", type=int, default=160, help="row blocks the CPU oracle is timed on")
-    ap.add_argument("--ref-rows", type=int, default=4, help="row blocks per step of the reference arm")
+    ap.add_argument("--ref-rows", type=int, default=12, help="row blocks per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only-topk", action="store_true", help="run only the stand-alone ranking kernel")
     ap.add_argument("--schedule-loop", action="store_true",
