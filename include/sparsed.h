@@ -38,7 +38,7 @@ extern "C" {
 typedef enum sparsed_status {
   SPARSED_OK = 0,
   SPARSED_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, heads_q % heads_kv != 0, ... */
-  SPARSED_ERR_UNSUPPORTED = 2,    /* head_dim != 128, block_size not in {64,128}, too many blocks */
+  SPARSED_ERR_UNSUPPORTED = 2,    /* head_dim != 128, block_size not in {32,64,128}, too many blocks */
   SPARSED_ERR_ALIGNMENT = 3,      /* seq_len or prefill_len not a multiple of block_size; pointer/stride alignment */
   SPARSED_ERR_WORKSPACE = 4,      /* workspace missing or too small */
   SPARSED_ERR_PATTERN = 5,        /* pattern arrays missing, too small, or inconsistent with the shape */
@@ -68,7 +68,7 @@ typedef struct sparsed_shape {
 } sparsed_shape;
 
 typedef struct sparsed_select_params {
-  int32_t block_size;  /* 64 or 128 */
+  int32_t block_size;  /* 32, 64 or 128 (the paper uses 32 for short and 128 for long contexts) */
   int32_t prefill_len; /* p of Eq. 6: keys [0,p) are prefill, [p,seq_len) generation; multiple of block_size */
   double keep_ratio;   /* rho in (0,1] */
   int32_t rounding;    /* 0: kept = ceil(rho * blocks in region) (default), 1: floor; at least 1 */
@@ -133,8 +133,8 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
  *                               probability mass a row puts on a tile), ranks it as
  *                               sparsed_select_pattern does (Eq. 5 / Eq. 6) and writes the CSR
  *                               pattern; scores_out_or_null optionally receives A'.
- * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; seq_len <= 131072 for
- * the selection (UNSUPPORTED beyond). Both buffers are caller-owned device memory.
+ * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; the selection needs
+ * seq_len <= 131072 and block_size 64 or 128 (the statistics are per 64 keys; UNSUPPORTED otherwise). Both buffers are caller-owned device memory.
  */
 sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, size_t *out_bytes); /* host only */
 sparsed_status sparsed_attn_full_stats(const sparsed_shape *shape, const void *q, const void *k, const void *v,

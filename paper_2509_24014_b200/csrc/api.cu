@@ -122,7 +122,7 @@ sparsed_status check_shape(const sparsed_shape* s, bool need_v_o, Resolved* r) {
 
 sparsed_status kept_counts(const sparsed_select_params* sp, int nb, int* pb, int* k_pre, int* k_gen) {
   if (sp == nullptr) return SPARSED_ERR_INVALID_ARG;
-  if (sp->block_size != 64 && sp->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (sp->block_size != 32 && sp->block_size != 64 && sp->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (!(sp->keep_ratio > 0.0) || !(sp->keep_ratio <= 1.0)) return SPARSED_ERR_INVALID_ARG;
   if (sp->rounding != 0 && sp->rounding != 1) return SPARSED_ERR_INVALID_ARG;
   if (sp->prefill_len < 0) return SPARSED_ERR_INVALID_ARG;
@@ -221,7 +221,7 @@ int32_t sparsed_schedule_mode(int32_t step_1based, int32_t total_steps, double s
 sparsed_status sparsed_kept_per_row(const sparsed_select_params* params, int32_t seq_len, int32_t* k_pre,
                                     int32_t* k_gen) {
   if (params == nullptr || k_pre == nullptr || k_gen == nullptr || seq_len < 1) return SPARSED_ERR_INVALID_ARG;
-  if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
   int pb = 0, a = 0, b = 0;
   sparsed_status st = kept_counts(params, seq_len / params->block_size, &pb, &a, &b);
@@ -243,7 +243,7 @@ sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape* shape, c
       return SPARSED_OK;
     case SPARSED_OP_SELECT_PATTERN: {
       if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
-      if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+      if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
       if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
       if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
       const size_t nb = static_cast<size_t>(shape->seq_len / params->block_size);
@@ -321,14 +321,15 @@ sparsed_status sparsed_select_from_stats(const sparsed_shape* shape, const spars
                                          float* scores_out_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
   if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
-  if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
   const int nb = shape->seq_len / params->block_size;
   int pb = 0, k_pre = 0, k_gen = 0;
   sparsed_status st = kept_counts(params, nb, &pb, &k_pre, &k_gen);
   if (st != SPARSED_OK) return st;
   if (lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
-  if (shape->seq_len > 131072) return SPARSED_ERR_UNSUPPORTED;
+  // the recorded statistics are per 64 keys: 32-key blocks need sparsed_select_pattern
+  if (shape->seq_len > 131072 || params->block_size == 32) return SPARSED_ERR_UNSUPPORTED;
   if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
     return st;
   if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
@@ -358,7 +359,7 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   if (q == nullptr || k == nullptr || v == nullptr || o == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SPARSED_ERR_ALIGNMENT;
   if (pattern == nullptr || pattern->row_ptr == nullptr || pattern->col_idx == nullptr) return SPARSED_ERR_PATTERN;
-  if (pattern->block_size != 64 && pattern->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (pattern->block_size != 32 && pattern->block_size != 64 && pattern->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (pattern->batch != shape->batch || pattern->heads_q != shape->heads_q || pattern->num_blocks < 1 ||
       static_cast<int64_t>(pattern->num_blocks) * pattern->block_size != shape->seq_len)
     return SPARSED_ERR_PATTERN;
@@ -367,8 +368,9 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   const int bs = pattern->block_size;
   CUtensorMap tq, tk, tv;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, bs)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 64)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 64)) != SPARSED_OK) return st;
+  const int kv_box = bs < 64 ? bs : 64;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, kv_box)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, kv_box)) != SPARSED_OK) return st;
   AttnParams p;
   p.o = o;
   p.o_stride_b = rs.o[0];
@@ -407,7 +409,7 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   sparsed_status st = check_shape(shape, false, &rs);
   if (st != SPARSED_OK) return st;
   if (params == nullptr) return SPARSED_ERR_INVALID_ARG;
-  if (params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
   const int nb = shape->seq_len / params->block_size;
   int pb = 0, k_pre = 0, k_gen = 0;
@@ -418,7 +420,7 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
     return st;
   // With few enough blocks per row the pooled-scoring kernel ranks each block-row in its own
   // tail; A' then goes to memory only if the caller asked for it.
-  const bool fused = nb <= kFusedTopkMaxBlocks;
+  const bool fused = nb <= kFusedTopkMaxBlocks && params->block_size != 32;
   const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
   const size_t score_bytes = round_up(bh * nb * nb * 4, 256);
   const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
@@ -467,7 +469,7 @@ sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int3
                                             int32_t sink_blocks, int32_t window_blocks, sparsed_pattern* out,
                                             void* cuda_stream) {
   if (batch < 1 || heads_q < 1 || num_blocks < 1 || sink_blocks < 0 || window_blocks < 1) return SPARSED_ERR_INVALID_ARG;
-  if (block_size != 64 && block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (block_size != 32 && block_size != 64 && block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (num_blocks > 16384) return SPARSED_ERR_UNSUPPORTED;
   if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
   const int sink = sink_blocks < num_blocks ? sink_blocks : num_blocks;

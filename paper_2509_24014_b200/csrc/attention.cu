@@ -57,7 +57,7 @@ struct AttnSmem {
 };
 
 // kSparse : walk the CSR list instead of all keys.  kBlock : keys per pattern block (sparse).
-// kRowsQ  : valid query rows per tile (64 or 128; the UMMA tile is always 128 rows).
+// kRowsQ  : valid query rows per tile (32, 64 or 128; the UMMA tile is always 128 rows).
 template <bool kSparse, int kBlock, int kRowsQ>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -72,7 +72,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
-  constexpr int kTilesPerBlock = kBlock / kTileN;
+  constexpr int kTilesPerBlock = kBlock >= kTileN ? kBlock / kTileN : 1;   // 128-key block: two tiles
+  constexpr int kBlocksPerTile = kBlock >= kTileN ? 1 : kTileN / kBlock;   // 32-key blocks: two per tile
 
   // ---- work item -----------------------------------------------------------------------
   const int q_tile = blockIdx.x % p.num_q_tiles;
@@ -82,11 +83,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const int kv_head = head / p.group;
   const int q_row0 = q_tile * kRowsQ;
 
-  int list_begin = 0, num_tiles;
+  int list_begin = 0, list_len = 0, num_tiles;
   if constexpr (kSparse) {
     const int r = bh * p.num_q_tiles + q_tile;
     list_begin = __ldg(p.row_ptr + r);
-    num_tiles = (__ldg(p.row_ptr + r + 1) - list_begin) * kTilesPerBlock;
+    list_len = __ldg(p.row_ptr + r + 1) - list_begin;
+    num_tiles = kBlocksPerTile == 1 ? list_len * kTilesPerBlock : (list_len + kBlocksPerTile - 1) / kBlocksPerTile;
   } else {
     num_tiles = (p.seq_len + kTileN - 1) / kTileN;
   }
@@ -117,6 +119,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     fence_proxy_async_smem();
   }
+  if constexpr (kBlocksPerTile > 1) {
+    // a tile may be half filled (odd list): its other half is multiplied by P = 0, so it has to
+    // hold finite numbers from the start
+    uint4* z = reinterpret_cast<uint4*>(&sm.kv[0][0][0]);
+    constexpr int n16 = kSlots * 2 * kTileN * 64 * 2 / 16;
+    for (int i = tid; i < n16; i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+  }
   if (warp == 5) {
     tmem_alloc(&sm.tmem_base, kTmemCols);
     tmem_relinquish();
@@ -145,13 +155,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       TL_DECL(2)
       bool ok = true;
       for (int t = 0; ok && t < num_tiles; ++t) {
-        int kv_row0;
-        if constexpr (kSparse) {
+        int kv_row0, kv_row1 = 0, blocks_here = 1;
+        if constexpr (!kSparse) {
+          kv_row0 = t * kTileN;
+        } else if constexpr (kBlocksPerTile == 1) {
           if (t % kTilesPerBlock == 0) block_id = __ldg(p.col_idx + list_begin + t / kTilesPerBlock);
           kv_row0 = block_id * kBlock + (t % kTilesPerBlock) * kTileN;
         } else {
-          kv_row0 = t * kTileN;
+          // two 32-key blocks side by side in one 64-key tile; an odd list leaves the last tile half filled
+          kv_row0 = __ldg(p.col_idx + list_begin + 2 * t) * kBlock;
+          if (2 * t + 1 < list_len) {
+            kv_row1 = __ldg(p.col_idx + list_begin + 2 * t + 1) * kBlock;
+            blocks_here = 2;
+          }
         }
+        (void)block_id;
         // load 2t (K_t) and load 2t+1 (V_t); a slot is reused every kSlots loads
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
@@ -164,10 +182,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             if (!ok) break;
           }
           if (elect_one_sync()) {
-            mbar_expect_tx(&sm.kv_full[slot], kTileN * kHeadDim * 2);
             const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
-            tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
-            tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+            if constexpr (kBlocksPerTile == 1) {
+              mbar_expect_tx(&sm.kv_full[slot], kTileN * kHeadDim * 2);
+              tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
+              tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+            } else {
+              // tensor-map boxes are 32 rows here; block b of the tile lands at rows 32 b
+              mbar_expect_tx(&sm.kv_full[slot], blocks_here * kBlock * kHeadDim * 2);
+              tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
+              tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+              if (blocks_here == 2) {
+                tma_load_4d(sm.kv[slot][0] + kBlock * 64, tm, &sm.kv_full[slot], 0, kv_row1, kv_head, batch);
+                tma_load_4d(sm.kv[slot][1] + kBlock * 64, tm, &sm.kv_full[slot], 64, kv_row1, kv_head, batch);
+              }
+            }
           }
           __syncwarp();
         }
@@ -272,8 +301,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tmem_ld32(tS + 32, r1);
       tmem_wait_ld();
       TL(3);
-      if constexpr (!kSparse) {
-        const int valid_cols = p.seq_len - t * kTileN;  // only the last tile can be ragged
+      if constexpr (!kSparse || kBlocksPerTile > 1) {
+        // only the last tile can be ragged: the tail of the sequence (dense) or an odd block list
+        const int valid_cols = kSparse ? (list_len - kBlocksPerTile * t) * kBlock : p.seq_len - t * kTileN;
         if (valid_cols < kTileN) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -444,11 +474,12 @@ cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, cons
   return launch<false, 128, 128>(tq, tk, tv, p, batch, stream);
 }
 
-// Tensor maps: Q box 64 x block_size rows, K and V boxes 64 x 64 rows.
+// Tensor maps: Q box 64 x block_size rows, K and V boxes 64 x min(64, block_size) rows.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
   if (block_size == 128) return launch<true, 128, 128>(tq, tk, tv, p, batch, stream);
-  return launch<true, 64, 64>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<true, 64, 64>(tq, tk, tv, p, batch, stream);
+  return launch<true, 32, 32>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed

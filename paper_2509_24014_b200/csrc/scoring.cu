@@ -177,6 +177,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         mbar_arrive(&sm.s_empty[buf]);
       } else {
         float half_sum[2] = {0.f, 0.f};
+        float quarter[4];
 #pragma unroll
         for (int c = 0; c < kTile / 32; ++c) {
           uint32_t r[32];
@@ -187,6 +188,25 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           for (int j = 0; j < 32; ++j)
             acc += tile_exp2<kScorePolyEvery>(fmaf(__uint_as_float(r[j]), scale_log2, -lse2), j);
           half_sum[c >> 1] += acc;
+          quarter[c] = acc;
+        }
+        if (p.block_size == 32) {
+          // 32-key blocks: a warp's 32 rows are one query block and each 32-column chunk one key
+          // block, so every warp finishes its own four scores (scores always go to memory here)
+          tc_fence_before();
+          mbar_arrive(&sm.s_empty[buf]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) quarter[c] += __shfl_xor_sync(0xffffffffu, quarter[c], off);
+          }
+          const int ib = q_tile * 4 + warp;
+          if (lane < 4 && ib < nb) {
+            const int jb = it * 4 + lane;
+            const float total = lane == 0 ? quarter[0] : (lane == 1 ? quarter[1] : (lane == 2 ? quarter[2] : quarter[3]));
+            if (jb < nb) p.scores[(static_cast<int64_t>(bh) * nb + ib) * nb + jb] = total * inv_area;
+          }
+          continue;
         }
         tc_fence_before();
         mbar_arrive(&sm.s_empty[buf]);

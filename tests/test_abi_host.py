@@ -60,12 +60,13 @@ def test_kept_per_row_matches_golden_table():
     assert sd.sparsed_kept_per_row(sd.make_params(128, 0.2, 4096), 8192) == (7, 7)
     assert sd.sparsed_kept_per_row(sd.make_params(128, 0.1, 16384), 32768) == (13, 13)
     assert sd.sparsed_kept_per_row(sd.make_params(128, 0.35, 0, rounding=1), 1280) == (0, 3)
+    assert sd.sparsed_kept_per_row(sd.make_params(32, 0.5, 352), 1024) == (6, 11)   # the short-context setting
 
 
 def test_argument_errors_are_status_codes(lib):
     with pytest.raises(sd.SparsedError) as e:
-        sd.sparsed_kept_per_row(sd.make_params(32, 0.3, 0), 1024)
-    assert e.value.status == 2                       # block size 32 unsupported
+        sd.sparsed_kept_per_row(sd.make_params(16, 0.3, 0), 1024)
+    assert e.value.status == 2                       # block size 16 unsupported
     with pytest.raises(sd.SparsedError) as e:
         sd.sparsed_kept_per_row(sd.make_params(128, 0.3, 0), 1000)
     assert e.value.status == 3                       # seq_len not a multiple of block_size
