@@ -390,7 +390,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         // which the pooled block scores are formed later without a second Q K^T pass
         const int row_g = q_row0 + tid;
         if (tid < kRowsQ && row_g < p.seq_len)
-          p.tile_lse[(static_cast<int64_t>(bh) * num_tiles + t) * p.seq_len + row_g] = m_used + __log2f(sum);
+          __stcs(p.tile_lse + (static_cast<int64_t>(bh) * num_tiles + t) * p.seq_len + row_g, m_used + __log2f(sum));  // streamed: read once, later
       }
       TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams 
       float v[kInFlight];
 #pragma unroll
       for (int u = 0; u < kInFlight; ++u)
-        v[u] = (row_valid && tt + u < n_here) ? __ldg(src + static_cast<int64_t>(c0 + tt + u) * L) : -INFINITY;
+        v[u] = (row_valid && tt + u < n_here) ? __ldcs(src + static_cast<int64_t>(c0 + tt + u) * L) : -INFINITY;
 #pragma unroll
       for (int u = 0; u < kInFlight; ++u)
         if (tt + u < n_here) sm.chunk[tt + u][tid] = fast_exp2(v[u] - lse2);

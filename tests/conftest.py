@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionstart(session):
+    """Build the CUDA library once if it is missing or older than its sources (nvcc cross-compiles
+    without a GPU). A failure here is not hidden: the tests that need the library then fail."""
+    try:
+        from paper_2509_24014_b200 import build
+        build.build_library()
+    except Exception as exc:  # pragma: no cover
+        print(f"[conftest] could not build libsparsed.so: {exc}")
