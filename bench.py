@@ -223,9 +223,14 @@ def run_ours(args, cfg):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    from paper_2509_24014_b200 import build as _build
     if int(os.environ.get("LOCAL_RANK", "0")) == 0:
-        from paper_2509_24014_b200 import build as _build
         _build.build_library()   # compiles only if the library is missing or older than its sources
+    else:
+        for _ in range(600):     # other ranks wait for rank 0's build instead of racing it
+            if not _build.is_stale():
+                break
+            time.sleep(0.5)
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
