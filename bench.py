@@ -154,6 +154,36 @@ def oracle_sparse_sample(cfg, q, k, v, rp, ci, n_row_blocks, seed=0):
     return flops / t_total / 1e12, t_total, n_row_blocks, threads
 
 
+def oracle_stage_samples(cfg, q, k, v, n_row_blocks, seed=1):
+    """Times the oracle's other stages (full attention; pooled scoring + selection) on a seeded
+    sample of (head, query block) rows and extrapolates to the whole workload (the work per row
+    block is uniform). Returns a dict for the cpu_baseline record."""
+    from oracle import sparsed_oracle as orc
+    rng = np.random.default_rng(seed)
+    nb, bs = cfg.num_blocks, cfg.block_size
+    group = cfg.heads_q // cfg.heads_kv
+    pb = cfg.prefill_len // bs
+    h = int(rng.integers(0, cfg.heads_q))
+    qh = q[0, h].to(torch.float64).numpy()
+    kh = k[0, h // group].to(torch.float64).numpy()
+    vh = v[0, h // group].to(torch.float64).numpy()
+    blocks = [int(x) for x in rng.integers(0, nb, n_row_blocks)]
+    t0 = time.perf_counter()
+    for ib in blocks:
+        orc.head_full_rows(qh, kh, vh, slice(ib * bs, (ib + 1) * bs))
+    t_full = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for ib in blocks:
+        orc.select_row(orc.head_pooled_row(qh, kh, ib, bs), pb, cfg.keep_ratio)
+    t_sel = time.perf_counter() - t0
+    total_rows = cfg.batch * cfg.heads_q * nb
+    scale = total_rows / n_row_blocks
+    return {"rows_sampled": n_row_blocks, "rows_total": total_rows,
+            "attn_full": {"cpu_seconds_sample": t_full, "cpu_seconds_extrapolated": t_full * scale,
+                          "tflops": 4.0 * bs * cfg.seq_len * cfg.head_dim * n_row_blocks / t_full / 1e12},
+            "score_and_select": {"cpu_seconds_sample": t_sel, "cpu_seconds_extrapolated": t_sel * scale}}
+
+
 def run_reference(args, cfg):
     """The oracle as it stands, timed on the host cores, on bounded samples of the workload."""
     from oracle import sparsed_oracle as orc
@@ -427,7 +457,11 @@ def run_ours(args, cfg):
         cpu = {"value": val, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
                "sample": f"oracle masked attention (fp64 numpy) on {rows} seeded (head, query block) rows of "
                          f"{Hq * nb}, GPU-selected pattern, {secs:.1f} s; kept-block FLOPs / time",
-               "seconds": secs, "host_cpus": os.cpu_count()}
+               "seconds": secs, "host_cpus": os.cpu_count(),
+               "cpu_seconds_extrapolated": secs * (B * Hq * nb) / rows,
+               "gpu_ms": {"attn_full_stats": full_total / n, "select_from_stats": select_total / n,
+                          "attn_sparse": sparse_total / n},
+               "other_stages": oracle_stage_samples(cfg, hq, hk, hv, max(4, n_rows // 8))}
 
     qkvo_gb = 4 * q.numel() * 2 / 1e9
     loop = None
@@ -710,7 +744,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c4", choices=sorted(syn.CONFIGS))
-    ap.add_argument("--cpu-rows", type=int, default=160, help="row blocks the CPU oracle is timed on")
+    ap.add_argument("--cpu-rows", type=int, default=128, help="row blocks the CPU oracle is timed on")
     ap.add_argument("--ref-rows", type=int, default=12, help="row blocks per step of the reference arm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only-topk", action="store_true", help="run only the stand-alone ranking kernel")
