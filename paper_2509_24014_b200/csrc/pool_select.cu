@@ -8,9 +8,10 @@
 // puts on tile t, so A'[ib][jb] is the sum of that mass over the rows of block ib and the tiles
 // of block jb, divided by block_size^2.
 //
-// One CTA owns one 128-row query tile of one (batch, head): thread r owns row r. Statistics
-// are read coalesced (row-fastest layout), exponentiated, transposed through padded shared
-// memory in chunks of 128 tiles, and summed per tile in a fixed order (bitwise reproducible).
+// One CTA owns one 128-row query tile of one (batch, head). Statistics are read with 16-byte
+// loads (four consecutive rows of one tile; row-fastest layout), sixteen in flight per thread,
+// exponentiated, parked in shared memory in chunks of 64 tiles, and summed per tile and row half
+// in a fixed, bank-conflict-free order (bitwise reproducible).
 // The CTA then holds its block-row(s) of A' in shared memory, optionally writes them out, and
 // warp 0 ranks them (warp_select_row) and writes the CSR lists. HBM-bound:
 // 4 * L * ceil(L/64) bytes read per (batch, head).
@@ -22,23 +23,24 @@ namespace {
 
 constexpr int kRows = 128;
 constexpr int kChunk = 64;          // tiles per transposition chunk
+constexpr int kPitch = kRows + 4;   // floats per chunk row: keeps float4 stores aligned
 #ifndef SPARSED_POOL_IN_FLIGHT
 #define SPARSED_POOL_IN_FLIGHT 16
 #endif
-constexpr int kInFlight = SPARSED_POOL_IN_FLIGHT;  // loads each thread keeps in flight
+constexpr int kInFlight = SPARSED_POOL_IN_FLIGHT;  // 16-byte loads each thread keeps in flight
 constexpr int kMaxTiles = 2048;     // seq_len <= 131072
 
 // Shared memory (dynamic, sized for the actual sequence): the transposition chunk, the per-tile
 // mass of rows 0-63 / 64-127, the ordered keys of this CTA's block-row(s), the top-k histogram.
 struct PoolSmem {
-  float (*chunk)[kRows + 1];        // [tile in chunk][row], padded against bank conflicts
+  float* chunk;                     // [tile in chunk][kPitch]
   float* tile_sum[2];               // [row half][tile]
   uint32_t* keys[2];
   int* hist;
 };
 
 __host__ __device__ inline size_t pool_smem_bytes(int n_tiles, int nb) {
-  return sizeof(float) * kChunk * (kRows + 1) + sizeof(float) * 2 * n_tiles + sizeof(uint32_t) * 2 * nb +
+  return sizeof(float) * kChunk * kPitch + sizeof(float) * 2 * n_tiles + sizeof(uint32_t) * 2 * nb +
          sizeof(int) * 256;
 }
 
@@ -50,8 +52,8 @@ __global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams 
   PoolSmem sm;
   {
     float* f = reinterpret_cast<float*>(pool_smem_raw);
-    sm.chunk = reinterpret_cast<float (*)[kRows + 1]>(f);
-    f += kChunk * (kRows + 1);
+    sm.chunk = f;
+    f += kChunk * kPitch;
     sm.tile_sum[0] = f;
     sm.tile_sum[1] = f + n_tiles;
     f += 2 * n_tiles;
@@ -63,32 +65,53 @@ __global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams 
   const int num_q_tiles = (L + kRows - 1) / kRows;
   const int q_tile = blockIdx.x % num_q_tiles;
   const int bh = blockIdx.x / num_q_tiles;
-  const int row = q_tile * kRows + tid;
-  const bool row_valid = row < L;
-  const float lse2 = row_valid ? p.lse[static_cast<int64_t>(bh) * L + row] * 1.44269504088896341f : INFINITY;
-  const float* src = p.tile_lse + static_cast<int64_t>(bh) * n_tiles * L + row;
+  // Loading: lane l owns rows 4l..4l+3 of the query tile (one 16-byte load covers them), warp w
+  // takes tiles w, w+4, ... of the chunk. seq_len is a multiple of 32 here, so a group of four
+  // rows is valid or invalid as a whole and 16-byte aligned.
+  const int row4 = q_tile * kRows + lane * 4;
+  const bool rows_valid = row4 < L;
+  float4 lse2 = make_float4(INFINITY, INFINITY, INFINITY, INFINITY);
+  if (rows_valid) {
+    const float4 t = *reinterpret_cast<const float4*>(p.lse + static_cast<int64_t>(bh) * L + row4);
+    const float c = 1.44269504088896341f;
+    lse2 = make_float4(t.x * c, t.y * c, t.z * c, t.w * c);
+  }
+  const float* src = p.tile_lse + static_cast<int64_t>(bh) * n_tiles * L + row4;
 
   for (int c0 = 0; c0 < n_tiles; c0 += kChunk) {
     const int n_here = min(kChunk, n_tiles - c0);
-    // coalesced over rows; kInFlight loads in flight per thread
-    for (int tt = 0; tt < n_here; tt += kInFlight) {
-      float v[kInFlight];
+    for (int tt = warp; tt < n_here; tt += 4 * kInFlight) {
+      float4 v[kInFlight];
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u)
-        v[u] = (row_valid && tt + u < n_here) ? __ldcs(src + static_cast<int64_t>(c0 + tt + u) * L) : -INFINITY;
+      for (int u = 0; u < kInFlight; ++u) {
+        const int t = tt + 4 * u;
+        v[u] = (rows_valid && t < n_here)
+                   ? __ldcs(reinterpret_cast<const float4*>(src + static_cast<int64_t>(c0 + t) * L))
+                   : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      }
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u)
-        if (tt + u < n_here) sm.chunk[tt + u][tid] = fast_exp2(v[u] - lse2);
+      for (int u = 0; u < kInFlight; ++u) {
+        const int t = tt + 4 * u;
+        if (t < n_here) {
+          const float4 e = make_float4(fast_exp2(v[u].x - lse2.x), fast_exp2(v[u].y - lse2.y),
+                                       fast_exp2(v[u].z - lse2.z), fast_exp2(v[u].w - lse2.w));
+          *reinterpret_cast<float4*>(sm.chunk + t * kPitch + lane * 4) = e;
+        }
+      }
     }
     __syncthreads();
-    if (tid < n_here) {
-      float s0 = 0.f, s1 = 0.f;
+    {
+      // Summing: thread j < 64 adds rows 0-63 of tile j, thread j + 64 rows 64-127. Each thread
+      // starts at its own rotation of the 64 rows so that a warp's reads hit 32 different banks;
+      // the order is fixed per tile, so the result is reproducible.
+      const int j = tid & 63, half = tid >> 6;
+      if (j < n_here) {
+        const float* rowp = sm.chunk + j * kPitch + half * 64;
+        float acc = 0.f;
 #pragma unroll 8
-      for (int r = 0; r < 64; ++r) s0 += sm.chunk[tid][r];
-#pragma unroll 8
-      for (int r = 64; r < 128; ++r) s1 += sm.chunk[tid][r];
-      sm.tile_sum[0][c0 + tid] = s0;
-      sm.tile_sum[1][c0 + tid] = s1;
+        for (int r = 0; r < 64; ++r) acc += rowp[(r + 29 * j) & 63];
+        sm.tile_sum[half][c0 + j] = acc;
+      }
     }
     __syncthreads();
   }
