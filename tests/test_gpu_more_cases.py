@@ -1,0 +1,81 @@
+"""Further GPU-vs-oracle cases: a non-default softmax scale through every entry point, batch > 1 on the
+statistics path, and logits that keep outgrowing the running maximum inside the sparse kernel."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_24014_b200 as sd
+from oracle import sparsed_oracle as orc
+from paper_2509_24014_b200 import synthetic as syn
+from tests.parity_util import check_outputs, to_f64
+from tests.test_gpu_parity_configs import SCORE_ATOL, SCORE_RTOL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def test_custom_scale_and_batch_two_through_all_entry_points():
+    cfg = syn.AttnConfig("s", 2, 4, 2, 768, 128, 128, 0.4, 256, seed=81)
+    q, k, v = syn.make_qkv(cfg, DEV)
+    scale = 0.11
+    scale32 = float(np.float32(scale))
+    qd, kd, vd = to_f64(q), to_f64(k), to_f64(v)
+    B, Hq, L, _ = q.shape
+    nb = L // 128
+    ws = sd.new_workspace(1 << 22, DEV)
+    o = torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=DEV)
+    stats = sd.new_tile_stats(q)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, softmax_scale=scale)
+    o_ref, lse_ref = orc.attn_full(qd, kd, vd, scale=scale32)
+    check_outputs(o, o_ref, "scaled full")
+    np.testing.assert_allclose(to_f64(lse), lse_ref, atol=3e-5, rtol=3e-6)
+    params = sd.make_params(128, 0.4, 256)
+    kp, kg = sd.sparsed_kept_per_row(params, L)
+    a_ref = orc.pooled_scores(qd, kd, 128, scale=scale32)
+    results = []
+    for path in ("stats", "two_pass", "two_pass_own_lse"):
+        pat, rp_t, ci_t = sd.new_pattern(B, Hq, nb, kp + kg, DEV)
+        scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=DEV)
+        if path == "stats":
+            sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws, scores_out=scores)
+        else:
+            sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse if path == "two_pass" else None,
+                                      scores_out=scores, softmax_scale=scale)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(scores.cpu().numpy(), a_ref, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+        rp, ci = orc.select_blocks(scores.cpu().numpy(), 128, 256, 0.4)
+        np.testing.assert_array_equal(ci_t.cpu().numpy(), ci)
+        np.testing.assert_array_equal(rp_t.cpu().numpy(), rp)
+        results.append((pat, rp, ci, rp_t, ci_t))
+    pat, rp, ci, _, _ = results[0]
+    o_sp = torch.empty_like(q)
+    sd.sparsed_attn_sparse(q, k, v, o_sp, pat, ws, softmax_scale=scale)
+    torch.cuda.synchronize()
+    check_outputs(o_sp, orc.attn_sparse(qd, kd, vd, rp, ci, 128, scale=scale32), "scaled sparse")
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+
+
+@pytest.mark.parametrize("bs", [64, 128])
+def test_sparse_kernel_with_growing_maxima(bs):
+    # keys sorted so that each query's logits keep rising along its kept list: exercises the rescale path
+    cfg = syn.AttnConfig("g", 1, 2, 2, 1024, 128, bs, 1.0, 0, seed=82)
+    q, k, v = syn.make_qkv(cfg, DEV)
+    q = (q.float() * 30).to(torch.bfloat16)
+    order = torch.argsort(k[0, 0].float() @ q[0, 0].float().mean(0))
+    k = k[:, :, order].contiguous()
+    v = v[:, :, order].contiguous()
+    nb = 1024 // bs
+    lists = [list(range(r % 3, nb, 2 + r % 2)) for r in range(2 * nb)]
+    rp = np.cumsum([0] + [len(x) for x in lists]).astype(np.int32)
+    ci = np.concatenate(lists).astype(np.int32)
+    rp_d, ci_d = torch.from_numpy(rp).to(DEV), torch.from_numpy(ci).to(DEV)
+    o = torch.empty_like(q)
+    ws = sd.new_workspace(256, DEV)
+    sd.sparsed_attn_sparse(q, k, v, o, sd.pattern_from_csr(rp_d, ci_d, bs, nb, 1, 2), ws)
+    torch.cuda.synchronize()
+    ref = orc.attn_sparse(to_f64(q), to_f64(k), to_f64(v), rp, ci, bs)
+    d = np.abs(to_f64(o) - ref)
+    assert d.max() <= 2e-2 * max(1.0, np.abs(ref).max()) and d.mean() <= 2e-3
+    assert np.linalg.norm(d) / np.linalg.norm(ref) <= 1e-2
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
