@@ -232,6 +232,14 @@ sparsed_status sparsed_select_pattern_static(const sparsed_shape *shape, const s
                                              const void *q, const void *k, const float *lse_or_null,
                                              sparsed_pattern *out, void *cuda_stream);
 
+/*
+ * Self-test of the failure path (no paper counterpart): launches one warp that waits, with a short
+ * poll limit, on a barrier nothing completes. The wait gives up, the kernel returns normally, and
+ * the status word of `ws` then reads code 1, where 99 (sparsed_last_device_status returns
+ * SPARSED_ERR_DEVICE_TIMEOUT). Clear it with sparsed_workspace_init; the context stays usable.
+ */
+sparsed_status sparsed_selftest_wait_timeout(void *ws, size_t ws_bytes, void *cuda_stream);
+
 const char *sparsed_status_string(sparsed_status status);
 int32_t sparsed_last_cuda_error(void);
 

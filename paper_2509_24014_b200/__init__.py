@@ -6,5 +6,5 @@ from .binding import (  # noqa: F401
     sparsed_tile_stats_bytes, new_workspace, pattern_from_csr, sparsed_attn_full, sparsed_attn_sparse, sparsed_build_window_pattern,
     sparsed_kept_per_row, sparsed_last_device_status, sparsed_pattern_validate, sparsed_schedule_mode,
     sparsed_select_from_scores, sparsed_select_pattern, sparsed_select_pattern_static, sparsed_switch_step, sparsed_workspace_bytes,
-    sparsed_workspace_init,
+    sparsed_workspace_init, sparsed_selftest_wait_timeout, save_pattern, load_pattern,
 )

@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_workspace_init", "sparsed_pattern_validate", "sparsed_last_device_status",
     "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
     "sparsed_tile_stats_bytes", "sparsed_attn_full_stats", "sparsed_select_from_stats",
-    "sparsed_build_window_pattern",
+    "sparsed_build_window_pattern", "sparsed_selftest_wait_timeout",
 )
 
 
@@ -77,6 +77,7 @@ def load_library() -> ctypes.CDLL:
     lib.sparsed_select_pattern.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
     lib.sparsed_build_window_pattern.argtypes = [i32, i32, i32, i32, i32, i32, P(Pattern), vp]
+    lib.sparsed_selftest_wait_timeout.argtypes = [vp, sz, vp]
     lib.sparsed_tile_stats_bytes.argtypes = [P(Shape), P(sz)]
     lib.sparsed_attn_full_stats.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_from_stats.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
@@ -294,6 +295,32 @@ def sparsed_pattern_validate(pattern: Pattern, ws: torch.Tensor) -> bool:
     if st == 5:
         return False
     raise SparsedError(int(st), "sparsed_pattern_validate")
+
+
+def sparsed_selftest_wait_timeout(ws: torch.Tensor) -> None:
+    _check(load_library().sparsed_selftest_wait_timeout(ws.data_ptr(), ws.numel(), _stream(ws)),
+           "sparsed_selftest_wait_timeout")
+
+
+def save_pattern(path: str, pattern: Pattern, row_ptr: torch.Tensor, col_idx: torch.Tensor, **meta) -> None:
+    """Writes a selected pattern to an .npz file: the only state the method carries across denoising
+    steps, so a run can resume in its sparse phase without selecting again."""
+    import numpy as np
+    np.savez(path, row_ptr=row_ptr.cpu().numpy(), col_idx=col_idx.cpu().numpy()[: int(pattern.nnz)],
+             block_size=pattern.block_size, num_blocks=pattern.num_blocks, batch=pattern.batch,
+             heads_q=pattern.heads_q, **meta)
+
+
+def load_pattern(path: str, device):
+    """Reads a pattern written by save_pattern; returns (Pattern, row_ptr, col_idx, meta dict)."""
+    import numpy as np
+    z = np.load(path if str(path).endswith(".npz") else str(path) + ".npz")
+    row_ptr = torch.from_numpy(z["row_ptr"]).to(device=device, dtype=torch.int32)
+    col_idx = torch.from_numpy(z["col_idx"]).to(device=device, dtype=torch.int32)
+    pat = pattern_from_csr(row_ptr, col_idx, int(z["block_size"]), int(z["num_blocks"]), int(z["batch"]),
+                           int(z["heads_q"]))
+    meta = {k: z[k].item() for k in z.files if k not in ("row_ptr", "col_idx", "block_size", "num_blocks", "batch", "heads_q")}
+    return pat, row_ptr, col_idx, meta
 
 
 def sparsed_last_device_status(ws: torch.Tensor) -> Tuple[int, int]:

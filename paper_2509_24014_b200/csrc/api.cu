@@ -511,6 +511,14 @@ sparsed_status sparsed_pattern_validate(const sparsed_pattern* pattern, void* ws
   return host_flag == 0 ? SPARSED_OK : SPARSED_ERR_PATTERN;
 }
 
+sparsed_status sparsed_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  sparsed_status st = check_arch();
+  if (st != SPARSED_OK) return st;
+  cudaError_t e = launch_wait_timeout_selftest(static_cast<DeviceStatus*>(ws), 99, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
+}
+
 sparsed_status sparsed_last_device_status(void* ws, void* cuda_stream, int32_t* code, int32_t* where) {
   if (ws == nullptr) return SPARSED_ERR_WORKSPACE;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -80,6 +80,7 @@ cudaError_t launch_pool_select(const PoolParams& p, cudaStream_t stream);
 int64_t window_pattern_nnz_per_head(int nb, int sink, int half);
 cudaError_t launch_window_pattern(int32_t* row_ptr, int32_t* col_idx, int bh, int nb, int sink, int half,
                                   int per_head_nnz, cudaStream_t stream);
+cudaError_t launch_wait_timeout_selftest(DeviceStatus* status, int where, cudaStream_t stream);
 cudaError_t launch_pattern_validate(const int32_t* row_ptr, const int32_t* col_idx, int rows, int nb,
                                     int64_t capacity, int* bad_flag, cudaStream_t stream);
 

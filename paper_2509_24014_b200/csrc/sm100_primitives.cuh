@@ -77,8 +77,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` lives in shared memory: once any thread of the CTA
 // gave up, the others stop waiting too.  Returns false when the wait gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          DeviceStatus* status, int where) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+                                          DeviceStatus* status, int where, uint32_t limit = kSpinLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }

@@ -62,7 +62,27 @@ __global__ void pattern_validate_kernel(const int32_t* row_ptr, const int32_t* c
   if (bad) atomicExch(bad_flag, r + 1);
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete, with
+// a short poll limit, so the wait gives up, records {1, where} in the status word and the kernel
+// returns normally.
+__global__ void wait_timeout_selftest_kernel(DeviceStatus* status, int where, uint32_t limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  mbar_wait(&bar, 0, &abort_flag, status, where, limit);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(DeviceStatus* status, int where, cudaStream_t stream) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status, where, 1u << 12);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_topk_csr(const TopkParams& p, cudaStream_t stream) {
   if (p.rows <= 0) return cudaSuccess;
