@@ -41,11 +41,11 @@ METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at
 # summarised under profiles/; keyed by (kernel, workload). None where no capture exists.
 NCU_DRAM_TRAFFIC = {
     # profiles/ncu_dram_bytes_c4_step_kernels.md (1-pass capture on the full-size workload)
-    ("attn_kernel<dense>", "c4"): 2491732736 + 9090945024,
+    ("attn_dense_pair_kernel", "c4"): 2491732736 + 9090945024,
     ("pool_select_kernel", "c4"): 8599094272 + 3844864,
     ("attn_kernel<sparse>", "c4"): 1259826944 + 516607744,
     # profiles/ncu_full_c2_all_kernels.md, profiles/ncu_full_topk_c4.md
-    ("attn_kernel<dense>", "c2"): 201578496 + 163437056,
+    ("attn_dense_pair_kernel", "c2"): 201578496 + 163437056,
     ("pool_select_kernel", "c2"): 135333376 + 3458048,
     ("attn_kernel<sparse>", "c2"): 156412416 + 42705920,
     ("topk_csr_kernel", "c4"): 33585920,
@@ -433,7 +433,7 @@ def run_ours(args, cfg):
         r = tensor_roofline("score_kernel (two-pass selection, not in the step)", dense_flops(cfg) / 2, times[1:])
         return r
 
-    roof_dense = tensor_roofline("attn_kernel<dense>", dense_flops(cfg), full_ms)
+    roof_dense = tensor_roofline("attn_dense_pair_kernel", dense_flops(cfg), full_ms)
     roof_sparse = tensor_roofline("attn_kernel<sparse>", sparse_flops(cfg, nnz), sparse_ms)
     # selection = pooled-scoring kernel (a dense QK^T contraction, 2*L^2*D per head) + top-k/CSR kernel
     launches_per_step = 3
@@ -495,7 +495,7 @@ def run_ours(args, cfg):
                 "what": "pinned host Q,K,V -> device, sparsed_attn_sparse, O -> pinned host; chunks of 4 kv heads on 3 streams", "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": launches_per_step * n,
-        "launches_per_step": {"attn_kernel<dense> (+ tile statistics)": 1,
+        "launches_per_step": {"attn_dense_pair_kernel (+ tile statistics)": 1,
                               "pool_select_kernel (pooling + top-k + CSR)": 1, "attn_kernel<sparse>": 1},
         "clocks": clocks, "peaks": peaks, "schedule_loop": loop,
     }

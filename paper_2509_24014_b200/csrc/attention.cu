@@ -1,5 +1,6 @@
-// Dense bidirectional attention (Eq. 1 times V) and block-sparse attention (Eq. 3 / Eq. 4
-// times V) for head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a.
+// Block-sparse attention (Eq. 3 / Eq. 4 times V; the "Sparse Reusing" branch of Algorithm 1) for
+// head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a. (The same template can walk all key
+// tiles; dense attention has its own two-tiles-per-CTA kernel in attention_dense.cu.)
 //
 // One CTA owns one query tile of one (batch, head) and streams 64-key tiles through a
 // warp-specialised pipeline:
@@ -467,12 +468,6 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
 }
 
 }  // namespace
-
-// Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows.
-cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                              const AttnParams& p, int batch, cudaStream_t stream) {
-  return launch<false, 128, 128>(tq, tk, tv, p, batch, stream);
-}
 
 // Tensor maps: Q box 64 x block_size rows, K and V boxes 64 x min(64, block_size) rows.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
