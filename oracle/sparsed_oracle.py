@@ -16,6 +16,10 @@ What each function follows in the paper:
 * ``attn_sparse``       - Eq. 3 with the block mask of Eq. 4, times V.
 * ``switch_step`` / ``schedule_mode`` - "Skipping Sparse" and the branch of Algorithm 1.
 * ``sparsed_attention`` - Algorithm 1 as a whole for one call.
+* ``pooled_qk_scores``  - NOT the paper's scorer: the cheap estimate of A' that pools queries and
+                          keys per block before the softmax (the approximate-score family the
+                          introduction sets the method against). Kept to measure how much of the
+                          exact pattern such an estimate recovers.
 
 Readings where the paper is silent (each listed in the design notes):
 pooling is over post-softmax probabilities normalised over the whole row; the number of
@@ -26,7 +30,9 @@ reads key/value head h // (Hq // Hkv).
 
 Parity status: pinned by the CPU tests against closed forms, a brute-force
 materialised implementation, a library routine and invariants. The paper prints no
-worked numeric example, so no pin comes from a printed value.
+worked numeric example, so no pin comes from a printed value. ``pooled_qk_scores`` is pinned
+by the two cases in which the estimate is exact (block size 1: a library softmax; inputs
+constant inside every block: the exact A').
 
 All tensors are numpy arrays: q [B,Hq,L,D], k and v [B,Hkv,L,D], float64 holding the
 exactly widened bf16 inputs.
@@ -121,6 +127,31 @@ def pooled_scores(q, k, block_size: int, scale: Optional[float] = None) -> np.nd
         for h in range(Hq):
             for ib in range(nb):
                 out[b, h, ib] = head_pooled_row(q[b, h], k[b, h // group], ib, block_size, scale)
+    return out
+
+
+def pooled_qk_scores(q, k, block_size: int, scale: Optional[float] = None) -> np.ndarray:
+    """Estimate of A' [B,Hq,nb,nb] from block means (not in the paper; see the module header).
+
+    Query block i and key block j are replaced by the means of their rows; the estimate of the
+    block's pooled probability is softmax_j(scale * mean_q[i] . mean_k[j]) / block_size, which has
+    the row sums (1 / block_size) of the exact A' and equals it when every block is constant.
+    """
+    B, Hq, L, D = q.shape
+    if L % block_size:
+        raise ValueError("seq_len must be a multiple of block_size")
+    nb = L // block_size
+    group = Hq // k.shape[1]
+    sc = _scale(D, scale)
+    out = np.empty((B, Hq, nb, nb), dtype=np.float64)
+    for b in range(B):
+        for h in range(Hq):
+            q_mean = q[b, h].reshape(nb, block_size, D).mean(axis=1)
+            k_mean = k[b, h // group].reshape(nb, block_size, D).mean(axis=1)
+            z = sc * (q_mean @ k_mean.T)
+            z -= z.max(axis=1, keepdims=True)
+            e = np.exp(z)
+            out[b, h] = e / e.sum(axis=1, keepdims=True) / block_size
     return out
 
 

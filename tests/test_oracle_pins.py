@@ -135,6 +135,41 @@ def test_pooled_invariants():
     assert a3[0].argmax() == 3 and a3[0, 3] > 0.9 / bs
 
 
+# ------------------------------------------------------------------ block-mean estimate of A'
+def test_pooled_qk_estimate_is_a_library_softmax_at_block_size_one():
+    from scipy.special import softmax
+    L, D = 20, 6
+    q, k, _ = _qkv(2, 4, 2, L, D, 70, qscale=1.3)
+    est = orc.pooled_qk_scores(q, k, 1)
+    for b in range(2):
+        for h in range(4):
+            ref = softmax((q[b, h] @ k[b, h // 2].T) / math.sqrt(D), axis=1)
+            np.testing.assert_allclose(est[b, h], ref, rtol=1e-12, atol=1e-16)
+    # and a custom scale is applied to the logits, not to the probabilities
+    est2 = orc.pooled_qk_scores(q, k, 1, scale=0.37)
+    np.testing.assert_allclose(est2[1, 3], softmax(0.37 * (q[1, 3] @ k[1, 1].T), axis=1), rtol=1e-12)
+
+
+def test_pooled_qk_estimate_is_exact_for_block_constant_inputs_and_only_then():
+    L, bs, D = 48, 8, 5
+    nb = L // bs
+    qb, kb, _ = _qkv(1, 2, 1, nb, D, 71, qscale=1.7)
+    q = np.repeat(qb, bs, axis=2)
+    k = np.repeat(kb, bs, axis=2)
+    est = orc.pooled_qk_scores(q, k, bs)
+    np.testing.assert_allclose(est, orc.pooled_scores(q, k, bs), rtol=1e-12, atol=1e-18)
+    np.testing.assert_allclose(est.sum(axis=-1), 1.0 / bs, rtol=1e-13)
+    # one strong key hidden among weak ones of its block: the exact A' sees it, the mean washes it out
+    q2, k2, _ = _qkv(1, 1, 1, L, D, 72, qscale=0.05)
+    u = np.ones(D) / math.sqrt(D)
+    q2[0, 0] += 3.0 * u
+    k2[0, 0, 19] += 12.0 * u          # token 19 lies in key block 2
+    exact = orc.pooled_scores(q2, k2, bs)[0, 0]
+    approx = orc.pooled_qk_scores(q2, k2, bs)[0, 0]
+    assert (exact.argmax(axis=1) == 2).all() and (approx.argmax(axis=1) == 2).all()
+    assert exact[:, 2].min() > 0.99 / bs and approx[:, 2].max() < 0.7 / bs
+
+
 # ------------------------------------------------------------------ Eq. 5 / Eq. 6 (selection)
 def test_kept_blocks_table():
     for n, rho, kept in _rows("kept_blocks_table.txt"):
