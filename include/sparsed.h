@@ -55,6 +55,7 @@ typedef enum sparsed_status {
 #define SPARSED_OP_SELECT_FROM_SCORES 2
 #define SPARSED_OP_ATTN_SPARSE 3
 #define SPARSED_OP_PATTERN_VALIDATE 4
+#define SPARSED_OP_SELECT_POOLED_QK 5
 
 /* Schedule modes returned by sparsed_schedule_mode. */
 #define SPARSED_MODE_FULL 0
@@ -143,6 +144,26 @@ sparsed_status sparsed_attn_full_stats(const sparsed_shape *shape, const void *q
 sparsed_status sparsed_select_from_stats(const sparsed_shape *shape, const sparsed_select_params *params,
                                          const float *lse, const float *tile_stats, sparsed_pattern *out,
                                          float *scores_out_or_null, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Block-mean ESTIMATE of A' and the selection from it. NOT the paper's scorer: the paper pools the
+ * exact post-softmax probabilities; this is the cheaper kind of estimate (pool first, then score)
+ * that the introduction sets the method against, offered so that its recall of the exact pattern
+ * and its cost can be measured on the same inputs through the same selection (Eq. 5 / Eq. 6):
+ *   mean_q[i], mean_k[j] = means of the rows of query block i / key block j (fp32),
+ *   est[i][j] = softmax_j(softmax_scale * mean_q[i] . mean_k[j]) / block_size
+ * (rows sum to 1 / block_size like A'; equal to A' when every block is constant).
+ * q, k: device bf16, layouts and strides as for sparsed_attn_full (v/o strides ignored).
+ * out: caller-owned CSR buffers as for sparsed_select_pattern; scores_out_or_null optionally
+ * receives est (device fp32 [batch, heads_q, num_blocks, num_blocks]).
+ * Workspace: sparsed_workspace_bytes(SPARSED_OP_SELECT_POOLED_QK, shape, params) bytes (status
+ * block + the block means). block_size 32, 64 or 128; seq_len / block_size <= 1024
+ * (UNSUPPORTED beyond). Asynchronous on the stream; deterministic.
+ */
+sparsed_status sparsed_select_pattern_pooled_qk(const sparsed_shape *shape, const sparsed_select_params *params,
+                                                const void *q, const void *k, sparsed_pattern *out,
+                                                float *scores_out_or_null, void *ws, size_t ws_bytes,
+                                                void *cuda_stream);
 
 /*
  * Block-sparse attention, O = softmax((Q K^T + M_S) / sqrt(d)) V with M_S the 0 / -inf block

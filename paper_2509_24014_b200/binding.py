@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 STATUS_BYTES = 256
-OP_ATTN_FULL, OP_SELECT_PATTERN, OP_SELECT_FROM_SCORES, OP_ATTN_SPARSE, OP_PATTERN_VALIDATE = range(5)
+OP_ATTN_FULL, OP_SELECT_PATTERN, OP_SELECT_FROM_SCORES, OP_ATTN_SPARSE, OP_PATTERN_VALIDATE, OP_SELECT_POOLED_QK = range(6)
 MODE_FULL, MODE_FULL_AND_SELECT, MODE_SPARSE = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_workspace_init", "sparsed_pattern_validate", "sparsed_last_device_status",
     "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
     "sparsed_tile_stats_bytes", "sparsed_attn_full_stats", "sparsed_select_from_stats",
-    "sparsed_build_window_pattern", "sparsed_selftest_wait_timeout",
+    "sparsed_build_window_pattern", "sparsed_selftest_wait_timeout", "sparsed_select_pattern_pooled_qk",
 )
 
 
@@ -75,6 +75,7 @@ def load_library() -> ctypes.CDLL:
     P = ctypes.POINTER
     lib.sparsed_attn_full.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_pattern.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp, vp, sz, vp]
+    lib.sparsed_select_pattern_pooled_qk.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
     lib.sparsed_build_window_pattern.argtypes = [i32, i32, i32, i32, i32, i32, P(Pattern), vp]
     lib.sparsed_selftest_wait_timeout.argtypes = [vp, sz, vp]
@@ -207,6 +208,17 @@ def sparsed_select_pattern(q, k, params: SelectParams, pattern: Pattern, ws: tor
         lse.data_ptr() if lse is not None else None, ctypes.byref(pattern),
         scores_out.data_ptr() if scores_out is not None else None, ws.data_ptr(), ws.numel(), _stream(q)),
         "sparsed_select_pattern")
+
+
+def sparsed_select_pattern_pooled_qk(q, k, params: SelectParams, pattern: Pattern, ws: torch.Tensor,
+                                     scores_out: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                                     shape: Optional[Shape] = None) -> None:
+    """Selection from the block-mean estimate of A' (a contrast scorer, not the paper's)."""
+    shape = shape or make_shape(q, k, None, None, softmax_scale)
+    _check(load_library().sparsed_select_pattern_pooled_qk(
+        ctypes.byref(shape), ctypes.byref(params), q.data_ptr(), k.data_ptr(), ctypes.byref(pattern),
+        scores_out.data_ptr() if scores_out is not None else None, ws.data_ptr(), ws.numel(), _stream(q)),
+        "sparsed_select_pattern_pooled_qk")
 
 
 def sparsed_tile_stats_bytes(shape: Shape) -> int:

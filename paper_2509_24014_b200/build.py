@@ -9,7 +9,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsparsed.so")
-SOURCES = ["api.cu", "attention.cu", "attention_dense.cu", "scoring.cu", "topk.cu", "pool_select.cu", "patterns.cu"]
+SOURCES = ["api.cu", "attention.cu", "attention_dense.cu", "scoring.cu", "topk.cu", "pool_select.cu", "patterns.cu", "pooled_qk.cu"]
 HEADERS = ["internal.h", "sm100_primitives.cuh", "topk_device.cuh", os.path.join("..", "..", "include", "sparsed.h")]
 
 

@@ -252,6 +252,15 @@ sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape* shape, c
                    round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
       return SPARSED_OK;
     }
+    case SPARSED_OP_SELECT_POOLED_QK: {
+      if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
+      if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+      if (shape->batch < 1 || shape->heads_q < 1 || shape->heads_kv < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+      if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+      *out_bytes = SPARSED_STATUS_BYTES +
+                   pooled_qk_means_bytes(shape->batch, shape->heads_q, shape->heads_kv, shape->seq_len / params->block_size);
+      return SPARSED_OK;
+    }
     default:
       return SPARSED_ERR_INVALID_ARG;
   }
@@ -347,6 +356,54 @@ sparsed_status sparsed_select_from_stats(const sparsed_shape* shape, const spars
   pp.k_gen = k_gen;
   pp.bh = shape->batch * shape->heads_q;
   cudaError_t e = launch_pool_select(pp, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
+}
+
+sparsed_status sparsed_select_pattern_pooled_qk(const sparsed_shape* shape, const sparsed_select_params* params,
+                                                const void* q, const void* k, sparsed_pattern* out,
+                                                float* scores_out_or_null, void* ws, size_t ws_bytes,
+                                                void* cuda_stream) {
+  Resolved rs;
+  sparsed_status st = check_shape(shape, false, &rs);
+  if (st != SPARSED_OK) return st;
+  if (params == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (q == nullptr || k == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return SPARSED_ERR_ALIGNMENT;
+  if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  const int nb = shape->seq_len / params->block_size;
+  int pb = 0, k_pre = 0, k_gen = 0;
+  if ((st = kept_counts(params, nb, &pb, &k_pre, &k_gen)) != SPARSED_OK) return st;
+  if (nb > kPooledQkMaxBlocks) return SPARSED_ERR_UNSUPPORTED;
+  if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
+    return st;
+  size_t need = 0;
+  if ((st = sparsed_workspace_bytes(SPARSED_OP_SELECT_POOLED_QK, shape, params, &need)) != SPARSED_OK) return st;
+  if (ws == nullptr || ws_bytes < need) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_arch()) != SPARSED_OK) return st;
+  PooledQkParams p;
+  p.q = q;
+  p.k = k;
+  p.q_stride_b = rs.q[0];
+  p.q_stride_h = rs.q[1];
+  p.q_stride_t = rs.q[2];
+  p.k_stride_b = rs.k[0];
+  p.k_stride_h = rs.k[1];
+  p.k_stride_t = rs.k[2];
+  p.means = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + SPARSED_STATUS_BYTES);
+  p.scores = scores_out_or_null;
+  p.row_ptr = out->row_ptr;
+  p.col_idx = out->col_idx;
+  p.batch = shape->batch;
+  p.heads_q = shape->heads_q;
+  p.group = shape->heads_q / shape->heads_kv;
+  p.nb = nb;
+  p.block_size = params->block_size;
+  p.pb = pb;
+  p.k_pre = k_pre;
+  p.k_gen = k_gen;
+  p.scale_log2 = rs.scale_log2;
+  cudaError_t e = launch_pooled_qk_select(p, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 

@@ -67,6 +67,27 @@ struct TopkParams {
   int k_pre, k_gen;
 };
 
+// Parameters of the block-mean estimate of A' (not the paper's scorer) and the selection from it.
+struct PooledQkParams {
+  const void* q;           // bf16 [B,Hq,L,128]
+  const void* k;           // bf16 [B,Hkv,L,128]
+  int64_t q_stride_b, q_stride_h, q_stride_t;
+  int64_t k_stride_b, k_stride_h, k_stride_t;
+  float* means;            // fp32 scratch: [B,Hq,nb,128] then [B,Hkv,nb,128]
+  float* scores;           // fp32 [B,Hq,nb,nb] or null
+  int32_t* row_ptr;
+  int32_t* col_idx;
+  int batch, heads_q, group;
+  int nb, block_size;
+  int pb, k_pre, k_gen;
+  float scale_log2;
+};
+
+// Largest number of key blocks per row the block-mean selection kernel holds in shared memory.
+constexpr int kPooledQkMaxBlocks = 1024;
+
+size_t pooled_qk_means_bytes(int batch, int heads_q, int heads_kv, int nb);
+cudaError_t launch_pooled_qk_select(const PooledQkParams& p, cudaStream_t stream);
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,

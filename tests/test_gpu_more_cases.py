@@ -1,5 +1,6 @@
 """Further GPU-vs-oracle cases: a non-default softmax scale through every entry point, batch > 1 on the
-statistics path, and logits that keep outgrowing the running maximum inside the sparse kernel."""
+statistics path, logits that keep outgrowing the running maximum inside the sparse kernel, and the batched
+long-context settings."""
 import numpy as np
 import pytest
 import torch
@@ -79,3 +80,52 @@ def test_sparse_kernel_with_growing_maxima(bs):
     assert d.max() <= 2e-2 * max(1.0, np.abs(ref).max()) and d.mean() <= 2e-3
     assert np.linalg.norm(d) / np.linalg.norm(ref) <= 1e-2
     assert sd.sparsed_last_device_status(ws) == (0, 0)
+
+
+@pytest.mark.parametrize("batch,seq_len,gen_len", [(16, 4096, 128), (8, 8192, 128)])
+def test_batched_long_context_settings(batch, seq_len, gen_len):
+    """The batched long-context evaluation settings (Table 3: batch 16 at 4k and batch 8 at 8k, block 128,
+    rho = 0.3): the switch step's fused path on the whole batch, the oracle on rows sampled over every
+    batch index."""
+    bs, rho = 128, 0.3
+    prefill = seq_len - gen_len
+    cfg = syn.AttnConfig("batched", batch, 8, 4, seq_len, 128, bs, rho, prefill, seed=300 + batch)
+    q, k, v = syn.make_qkv(cfg, DEV)
+    B, Hq, L, _ = q.shape
+    nb, pb, group = L // bs, prefill // bs, 2
+    ws = sd.new_workspace(1 << 22, DEV)
+    o = torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=DEV)
+    stats = sd.new_tile_stats(q)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+    params = sd.make_params(bs, rho, prefill)
+    kp, kg = sd.sparsed_kept_per_row(params, L)
+    assert (kp, kg) == (orc.kept_per_region(pb, rho), orc.kept_per_region(nb - pb, rho))
+    pat, rp_t, ci_t = sd.new_pattern(B, Hq, nb, kp + kg, DEV)
+    scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=DEV)
+    sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws, scores_out=scores)
+    o_sp = torch.empty_like(q)
+    sd.sparsed_attn_sparse(q, k, v, o_sp, pat, ws)
+    torch.cuda.synchronize()
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+    assert pat.nnz == B * Hq * nb * (kp + kg)
+    rp, ci = rp_t.cpu().numpy(), ci_t.cpu().numpy()
+    # the selection is bit-exact on the GPU's own scores for every row of every batch element
+    rp_ref, ci_ref = orc.select_blocks(scores.cpu().numpy(), bs, prefill, rho)
+    np.testing.assert_array_equal(rp, rp_ref)
+    np.testing.assert_array_equal(ci, ci_ref)
+    rng = np.random.default_rng(batch)
+    for b in range(B):
+        h = int(rng.integers(Hq))
+        ib = int(rng.choice([0, pb - 1, pb, nb - 1, int(rng.integers(nb))]))
+        qh, kh, vh = to_f64(q[b, h]), to_f64(k[b, h // group]), to_f64(v[b, h // group])
+        rows = slice(ib * bs, (ib + 1) * bs)
+        o_ref, lse_ref = orc.head_full_rows(qh, kh, vh, rows)
+        check_outputs(o[b, h, rows], o_ref, f"batched full b{b} h{h} ib{ib}")
+        np.testing.assert_allclose(to_f64(lse[b, h, rows]), lse_ref, atol=3e-5, rtol=3e-6)
+        np.testing.assert_allclose(scores[b, h, ib].cpu().numpy(), orc.head_pooled_row(qh, kh, ib, bs),
+                                   rtol=SCORE_RTOL, atol=SCORE_ATOL)
+        r = (b * Hq + h) * nb + ib
+        kept = ci[rp[r]:rp[r + 1]]
+        check_outputs(o_sp[b, h, rows], orc.head_sparse_rows(qh, kh, vh, ib, kept, bs),
+                      f"batched sparse b{b} h{h} ib{ib}")
