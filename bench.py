@@ -740,6 +740,74 @@ def run_sweep(args, cfg):
                       "ablation_schedule_ms": ablation, "comparison_patterns": base}))
 
 
+def run_estimate_recall(args, cfg):
+    """The exact switch-step selection beside the block-mean estimate (pool Q and K first, then score; not the
+    paper's scorer) on the same inputs: time of each, how much of the exact pattern the estimate recovers
+    (by count and by A' mass) and the error each pattern leaves in the sparse output against full attention,
+    per planted head kind."""
+    import numpy as np
+    import paper_2509_24014_b200 as sd
+    from paper_2509_24014_b200 import pattern_metrics as pm
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    q, k, v = syn.make_qkv(cfg, dev)
+    B, Hq, L, D = q.shape
+    bs, nb = cfg.block_size, cfg.num_blocks
+    params = sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)
+    k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
+    o_full, o_sp = torch.empty_like(q), torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+    stats = sd.new_tile_stats(q)
+    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_POOLED_QK, sd.make_shape(q, k), params), dev)
+    scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=dev)
+    pat_x, rp_x, ci_x = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+    pat_e, rp_e, ci_e = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+
+    def timed(fn, reps=5):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = _ev(), _ev()
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+
+    sd.sparsed_attn_full_stats(q, k, v, o_full, lse, stats, ws)
+    exact_ms = timed(lambda: sd.sparsed_select_from_stats(q, k, params, lse, stats, pat_x, ws, scores_out=scores))
+    est_ms = timed(lambda: sd.sparsed_select_pattern_pooled_qk(q, k, params, pat_e, ws))
+    torch.cuda.synchronize()
+    a_exact = scores.cpu().numpy().reshape(B * Hq * nb, nb)
+    rpx, cix, rpe, cie = (t.cpu().numpy() for t in (rp_x, ci_x, rp_e, ci_e))
+    recall = pm.pattern_recall(rpx, cix, rpe, cie, nb).reshape(B, Hq, nb)
+    mass_x = pm.kept_mass(a_exact, rpx, cix).reshape(B, Hq, nb) * bs     # share of each row block's probability mass
+    mass_e = pm.kept_mass(a_exact, rpe, cie).reshape(B, Hq, nb) * bs
+
+    def out_err(pat):
+        sd.sparsed_attn_sparse(q, k, v, o_sp, pat, ws)
+        torch.cuda.synchronize()
+        num = torch.stack([(o_sp[:, h].float() - o_full[:, h].float()).norm() for h in range(Hq)])
+        den = torch.stack([o_full[:, h].float().norm() for h in range(Hq)])
+        return (num / den).cpu().numpy()
+
+    err_x, err_e = out_err(pat_x), out_err(pat_e)
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+    kinds = [kd[0] for kd in syn.head_kinds(cfg)]
+    by_kind = {}
+    for name in sorted(set(kinds)):
+        hs = [h for h in range(Hq) if kinds[h] == name]
+        by_kind[name] = {"heads": len(hs), "recall": float(recall[:, hs].mean()),
+                         "kept_mass_exact": float(mass_x[:, hs].mean()), "kept_mass_estimate": float(mass_e[:, hs].mean()),
+                         "sparse_vs_full_rel_err_exact": float(err_x[hs].mean()),
+                         "sparse_vs_full_rel_err_estimate": float(err_e[hs].mean())}
+    print(json.dumps({"workload": workload_name(cfg), "plant_norm": cfg.plant_norm,
+                      "select_from_stats_ms": exact_ms, "select_pooled_qk_ms": est_ms,
+                      "recall_of_exact_pattern": float(recall.mean()), "kept_mass_exact": float(mass_x.mean()),
+                      "kept_mass_estimate": float(mass_e.mean()), "sparse_vs_full_rel_err_exact": float(err_x.mean()),
+                      "sparse_vs_full_rel_err_estimate": float(err_e.mean()), "by_head_kind": by_kind}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -756,9 +824,17 @@ def main():
     ap.add_argument("--all-full", action="store_true", help="with --schedule-loop: also time all-full attention")
     ap.add_argument("--no-schedule-loop", action="store_true", help="skip the schedule-loop summary of the default run")
     ap.add_argument("--sweep", action="store_true", help="keep-ratio / isolation / ablation / comparison-pattern timings")
+    ap.add_argument("--estimate-recall", action="store_true",
+                    help="exact selection vs the block-mean estimate: time, recall, kept mass, output error")
+    ap.add_argument("--plant-norm", type=float, default=None,
+                    help="norm of the planted vectors (default 3: logit boost 0.8; 9 gives sharp attention)")
     args = ap.parse_args()
     cfg = syn.CONFIGS[args.config]
-    if args.sweep:
+    if args.plant_norm is not None:
+        cfg = cfg.with_(plant_norm=args.plant_norm)
+    if args.estimate_recall:
+        run_estimate_recall(args, cfg)
+    elif args.sweep:
         run_sweep(args, cfg)
     elif args.schedule_loop:
         run_schedule_loop(args, cfg)

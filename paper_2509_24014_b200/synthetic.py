@@ -46,6 +46,7 @@ class AttnConfig:
     step_noise: float = 0.0
     hidden: int = 0  # > 0: Q/K/V come from random projections of a hidden state of this width
     fixed_heads: Optional[Tuple[Tuple[str, ...], ...]] = None
+    plant_norm: float = 3.0  # L2 norm of the planted vectors: logit boost plant_norm^2 / sqrt(head_dim)
 
     @property
     def num_blocks(self) -> int:
@@ -67,9 +68,6 @@ CONFIGS: Dict[str, AttnConfig] = {
     "c5": AttnConfig("c5", 1, 32, 32, 32768, 128, 128, 0.1, 16384, seed=5, total_steps=256, skip=0.25,
                      layers=4, hidden=4096),
 }
-
-_PLANT_NORM = 3.0
-
 
 def _gen(device, *key: int) -> torch.Generator:
     g = torch.Generator(device=device)
@@ -107,9 +105,9 @@ def head_kinds(cfg: AttnConfig, layer: int = 0) -> List[Tuple]:
     return kinds
 
 
-def _direction(g: torch.Generator, shape, device) -> torch.Tensor:
+def _direction(g: torch.Generator, shape, device, norm: float) -> torch.Tensor:
     u = torch.randn(*shape, generator=g, device=device, dtype=torch.float32)
-    return u * (_PLANT_NORM / u.norm(dim=-1, keepdim=True))
+    return u * (norm / u.norm(dim=-1, keepdim=True))
 
 
 def _plant(cfg: AttnConfig, q: torch.Tensor, k: torch.Tensor, layer: int) -> None:
@@ -124,12 +122,12 @@ def _plant(cfg: AttnConfig, q: torch.Tensor, k: torch.Tensor, layer: int) -> Non
         if kind[0] == "band":
             w = kind[1]
             cells = (L + w - 1) // w
-            u = _direction(g, (cells, D), device)
+            u = _direction(g, (cells, D), device, cfg.plant_norm)
             cell = torch.arange(L, device=device) // w
             q[:, h] += u[cell]
             k[:, hk] += u[cell]
         elif kind[0] in ("sink", "sink+stripes", "stripes"):
-            a = _direction(g, (D,), device)
+            a = _direction(g, (D,), device, cfg.plant_norm)
             q[:, h] += a
             if kind[0] != "stripes":
                 k[:, hk, : kind[1]] += a
