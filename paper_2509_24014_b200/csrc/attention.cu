@@ -1,6 +1,6 @@
 // Block-sparse attention (Eq. 3 / Eq. 4 times V; the "Sparse Reusing" branch of Algorithm 1) for
-// head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a. (The same template can walk all key
-// tiles; dense attention has its own two-tiles-per-CTA kernel in attention_dense.cu.)
+// head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a. (Dense attention has its own
+// two-tiles-per-CTA kernel in attention_dense.cu.)
 //
 // One CTA owns one query tile of one (batch, head) and streams 64-key tiles through a
 // warp-specialised pipeline:
@@ -16,9 +16,9 @@
 //             logits may have outgrown it by more than 2^8 is the tile redone with the new
 //             maximum and O rescaled (after the previous P V has drained). Finally O is
 //             normalised and stored.
-// The dense kernel walks all key tiles; the sparse kernel walks the CSR list of its query
-// block (a 128-key block is two consecutive tiles). Two CTAs fit on one SM (112 KB of shared
-// memory and 256 tensor-memory columns each).
+// The tile index comes from the CSR list of the CTA's query block (a 128-key block is two
+// consecutive tiles, two 32-key blocks share one). Two CTAs fit on one SM (112 KB of shared memory
+// and 256 tensor-memory columns each).
 #include "internal.h"
 
 namespace sparsed {
@@ -57,9 +57,9 @@ struct AttnSmem {
   int abort_flag;
 };
 
-// kSparse : walk the CSR list instead of all keys.  kBlock : keys per pattern block (sparse).
-// kRowsQ  : valid query rows per tile (32, 64 or 128; the UMMA tile is always 128 rows).
-template <bool kSparse, int kBlock, int kRowsQ>
+// kBlock : keys per pattern block.
+// kRowsQ : valid query rows per tile (32, 64 or 128; the UMMA tile is always 128 rows).
+template <int kBlock, int kRowsQ>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
@@ -84,19 +84,36 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const int kv_head = head / p.group;
   const int q_row0 = q_tile * kRowsQ;
 
-  int list_begin = 0, list_len = 0, num_tiles;
-  if constexpr (kSparse) {
-    const int r = bh * p.num_q_tiles + q_tile;
-    list_begin = __ldg(p.row_ptr + r);
-    list_len = __ldg(p.row_ptr + r + 1) - list_begin;
-    num_tiles = kBlocksPerTile == 1 ? list_len * kTilesPerBlock : (list_len + kBlocksPerTile - 1) / kBlocksPerTile;
-  } else {
-    num_tiles = (p.seq_len + kTileN - 1) / kTileN;
-  }
+  const int r = bh * p.num_q_tiles + q_tile;
+  const int list_begin = __ldg(p.row_ptr + r);
+  const int list_len = __ldg(p.row_ptr + r + 1) - list_begin;
+  const int num_tiles =
+      kBlocksPerTile == 1 ? list_len * kTilesPerBlock : (list_len + kBlocksPerTile - 1) / kBlocksPerTile;
 
   // ---- set-up --------------------------------------------------------------------------
+  // The producer warp starts the two loads nothing else depends on before the CTA-wide set-up has
+  // finished: the Q tile (through a barrier it initialises itself) and the first 32 ids of the list.
+  int list_ids = 0;  // warp 4: lane i holds col_idx[list_begin + 32 * chunk + i] of the current chunk
+  if (warp == 4) {
+    if ((tid & 31) == 0) {
+      mbar_init(&sm.q_full, 1);
+      mbar_fence_init();
+    }
+    __syncwarp();
+    if (num_tiles > 0) {
+      if (elect_one_sync()) {
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        mbar_expect_tx(&sm.q_full, kRowsQ * kHeadDim * 2);
+        tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
+        tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
+      }
+      __syncwarp();
+      if ((tid & 31) < list_len) list_ids = __ldg(p.col_idx + list_begin + (tid & 31));
+    }
+  }
   if (tid == 0) {
-    mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(&sm.kv_full[s], 1);
       mbar_init(&sm.kv_empty[s], 1);
@@ -143,34 +160,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if (warp == 4) {
     // =============================== TMA producer =======================================
     if (num_tiles > 0) {
-      if (elect_one_sync()) {
-        tma_prefetch_desc(&tm_q);
-        tma_prefetch_desc(&tm_k);
-        tma_prefetch_desc(&tm_v);
-        mbar_expect_tx(&sm.q_full, kRowsQ * kHeadDim * 2);
-        tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
-        tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
-      }
-      __syncwarp();
-      int block_id = 0;
+      const int lane = tid & 31;
       TL_DECL(2)
       bool ok = true;
       for (int t = 0; ok && t < num_tiles; ++t) {
+        // list entry of this tile's (first) block; ids are fetched 32 at a time, one per lane
+        const int e = kBlocksPerTile == 1 ? t / kTilesPerBlock : kBlocksPerTile * t;
+        if (e > 0 && (e & 31) == 0 && (kBlocksPerTile > 1 || t % kTilesPerBlock == 0))
+          list_ids = (e + lane < list_len) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
         int kv_row0, kv_row1 = 0, blocks_here = 1;
-        if constexpr (!kSparse) {
-          kv_row0 = t * kTileN;
-        } else if constexpr (kBlocksPerTile == 1) {
-          if (t % kTilesPerBlock == 0) block_id = __ldg(p.col_idx + list_begin + t / kTilesPerBlock);
-          kv_row0 = block_id * kBlock + (t % kTilesPerBlock) * kTileN;
+        if constexpr (kBlocksPerTile == 1) {
+          kv_row0 = __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock + (t % kTilesPerBlock) * kTileN;
         } else {
           // two 32-key blocks side by side in one 64-key tile; an odd list leaves the last tile half filled
-          kv_row0 = __ldg(p.col_idx + list_begin + 2 * t) * kBlock;
-          if (2 * t + 1 < list_len) {
-            kv_row1 = __ldg(p.col_idx + list_begin + 2 * t + 1) * kBlock;
+          kv_row0 = __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock;
+          const int second = __shfl_sync(0xffffffffu, list_ids, (e + 1) & 31);
+          if (e + 1 < list_len) {
+            kv_row1 = second * kBlock;
             blocks_here = 2;
           }
         }
-        (void)block_id;
         // load 2t (K_t) and load 2t+1 (V_t); a slot is reused every kSlots loads
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
@@ -302,9 +311,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tmem_ld32(tS + 32, r1);
       tmem_wait_ld();
       TL(3);
-      if constexpr (!kSparse || kBlocksPerTile > 1) {
-        // only the last tile can be ragged: the tail of the sequence (dense) or an odd block list
-        const int valid_cols = kSparse ? (list_len - kBlocksPerTile * t) * kBlock : p.seq_len - t * kTileN;
+      if constexpr (kBlocksPerTile > 1) {
+        // only the last tile can be ragged: an odd block list leaves its second half empty
+        const int valid_cols = (list_len - kBlocksPerTile * t) * kBlock;
         if (valid_cols < kTileN) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -386,13 +395,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       }
       l += sum;
-      if (p.tile_lse != nullptr) {
-        // switch step: keep log2 of this tile's share of the row's softmax denominator, from
-        // which the pooled block scores are formed later without a second Q K^T pass
-        const int row_g = q_row0 + tid;
-        if (tid < kRowsQ && row_g < p.seq_len)
-          __stcs(p.tile_lse + (static_cast<int64_t>(bh) * num_tiles + t) * p.seq_len + row_g, m_used + __log2f(sum));  // streamed: read once, later
-      }
       TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();
@@ -401,7 +403,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       TL(5);
     }
 
-    // ---- epilogue: O / l -> bf16 -> global; LSE ----------------------------------------
+    // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
     if (ok && num_tiles > 0) ok = mbar_wait(&sm.o_full, 0, &sm.abort_flag, p.status, 31);
     tc_fence_after();
     const int row_in_tile = tid;
@@ -433,10 +435,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       }
     }
-    if (p.lse != nullptr && row_valid) {
-      const float lse = (num_tiles > 0) ? (m_used + log2f(l)) * 0.69314718055994531f : -INFINITY;
-      p.lse[static_cast<int64_t>(bh) * p.seq_len + row] = lse;
-    }
   }
 
   // ---- teardown ------------------------------------------------------------------------
@@ -448,10 +446,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <bool kSparse, int kBlock, int kRowsQ>
+template <int kBlock, int kRowsQ>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kSparse, kBlock, kRowsQ>;
+  auto kernel = attn_kernel<kBlock, kRowsQ>;
   const int smem = static_cast<int>(sizeof(AttnSmem));
   static bool configured[64] = {};  // per template instantiation and device
   int dev = 0;
@@ -472,9 +470,9 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
 // Tensor maps: Q box 64 x block_size rows, K and V boxes 64 x min(64, block_size) rows.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<true, 128, 128>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<true, 64, 64>(tq, tk, tv, p, batch, stream);
-  return launch<true, 32, 32>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<128, 128>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<64, 64>(tq, tk, tv, p, batch, stream);
+  return launch<32, 32>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed
