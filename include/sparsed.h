@@ -56,6 +56,7 @@ typedef enum sparsed_status {
 #define SPARSED_OP_ATTN_SPARSE 3
 #define SPARSED_OP_PATTERN_VALIDATE 4
 #define SPARSED_OP_SELECT_POOLED_QK 5
+#define SPARSED_OP_ATTENTION_STEP 6
 
 /* Schedule modes returned by sparsed_schedule_mode. */
 #define SPARSED_MODE_FULL 0
@@ -185,6 +186,30 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape *shape, const sparsed_pat
  */
 int32_t sparsed_schedule_mode(int32_t step_1based, int32_t total_steps, double skip);
 int32_t sparsed_switch_step(int32_t total_steps, double skip);
+
+/*
+ * Algorithm 1 for one attention call of denoising step `step_1based` (1-based) of `total_steps`:
+ *   steps before the switch step  : full attention (Eq. 1)                  -> *mode = SPARSED_MODE_FULL
+ *   the switch step               : full attention, then the pattern is selected from that very pass
+ *                                   (A' = avgpool(A), Eq. 5 / Eq. 6) and written to `pattern`
+ *                                                                            -> SPARSED_MODE_FULL_AND_SELECT
+ *   later steps                   : block-sparse attention (Eq. 3 / Eq. 4) with `pattern` as the
+ *                                   switch step left it ("Sparse Reusing")   -> SPARSED_MODE_SPARSE
+ * The same calls as sparsed_attn_full / sparsed_attn_full_stats + sparsed_select_from_stats /
+ * sparsed_attn_sparse, chosen by sparsed_schedule_mode; where the statistics path does not apply
+ * (block_size 32, seq_len > 131072) the switch step selects with sparsed_select_pattern instead.
+ * q, k, v, o: device bf16 as for sparsed_attn_full. pattern: caller-owned CSR buffers sized as for
+ * sparsed_select_pattern, written at the switch step and only read afterwards; the caller keeps it
+ * (one per layer) across steps. ws: device workspace, zeroed status block first; the switch step
+ * needs sparsed_workspace_bytes(SPARSED_OP_ATTENTION_STEP, shape, params) bytes (row statistics of
+ * the full pass: 4 * seq_len * ceil(seq_len / 64) bytes per head), every other step only
+ * SPARSED_STATUS_BYTES. mode_out_or_null (host) receives the mode that ran. Errors as for the calls
+ * it makes; INVALID_ARG for a step outside 1..total_steps or skip outside [0, 1]. Asynchronous.
+ */
+sparsed_status sparsed_attention_step(const sparsed_shape *shape, const sparsed_select_params *params,
+                                      int32_t step_1based, int32_t total_steps, double skip, const void *q,
+                                      const void *k, const void *v, void *o, sparsed_pattern *pattern, void *ws,
+                                      size_t ws_bytes, void *cuda_stream, int32_t *mode_out_or_null);
 
 /*
  * Number of key blocks kept per query block in the prefill and generation regions

@@ -15,7 +15,8 @@ import torch
 from . import build as _build
 
 STATUS_BYTES = 256
-OP_ATTN_FULL, OP_SELECT_PATTERN, OP_SELECT_FROM_SCORES, OP_ATTN_SPARSE, OP_PATTERN_VALIDATE, OP_SELECT_POOLED_QK = range(6)
+(OP_ATTN_FULL, OP_SELECT_PATTERN, OP_SELECT_FROM_SCORES, OP_ATTN_SPARSE, OP_PATTERN_VALIDATE, OP_SELECT_POOLED_QK,
+ OP_ATTENTION_STEP) = range(7)
 MODE_FULL, MODE_FULL_AND_SELECT, MODE_SPARSE = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
@@ -25,6 +26,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
     "sparsed_tile_stats_bytes", "sparsed_attn_full_stats", "sparsed_select_from_stats",
     "sparsed_build_window_pattern", "sparsed_selftest_wait_timeout", "sparsed_select_pattern_pooled_qk",
+    "sparsed_attention_step",
 )
 
 
@@ -76,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     lib.sparsed_attn_full.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_pattern.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_pattern_pooled_qk.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
+    lib.sparsed_attention_step.argtypes = [P(Shape), P(SelectParams), i32, i32, ctypes.c_double, vp, vp, vp, vp,
+                                           P(Pattern), vp, sz, vp, P(i32)]
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
     lib.sparsed_build_window_pattern.argtypes = [i32, i32, i32, i32, i32, i32, P(Pattern), vp]
     lib.sparsed_selftest_wait_timeout.argtypes = [vp, sz, vp]
@@ -219,6 +223,19 @@ def sparsed_select_pattern_pooled_qk(q, k, params: SelectParams, pattern: Patter
         ctypes.byref(shape), ctypes.byref(params), q.data_ptr(), k.data_ptr(), ctypes.byref(pattern),
         scores_out.data_ptr() if scores_out is not None else None, ws.data_ptr(), ws.numel(), _stream(q)),
         "sparsed_select_pattern_pooled_qk")
+
+
+def sparsed_attention_step(q, k, v, o, params: SelectParams, step_1based: int, total_steps: int, skip: float,
+                           pattern: Pattern, ws: torch.Tensor, softmax_scale: float = 0.0,
+                           shape: Optional[Shape] = None) -> int:
+    """Algorithm 1 for one attention call of one denoising step; returns the mode that ran."""
+    shape = shape or make_shape(q, k, v, o, softmax_scale)
+    mode = ctypes.c_int32(-1)
+    _check(load_library().sparsed_attention_step(
+        ctypes.byref(shape), ctypes.byref(params), int(step_1based), int(total_steps), float(skip), q.data_ptr(),
+        k.data_ptr(), v.data_ptr(), o.data_ptr(), ctypes.byref(pattern), ws.data_ptr(), ws.numel(), _stream(q),
+        ctypes.byref(mode)), "sparsed_attention_step")
+    return int(mode.value)
 
 
 def sparsed_tile_stats_bytes(shape: Shape) -> int:

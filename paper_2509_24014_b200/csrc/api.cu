@@ -146,6 +146,11 @@ sparsed_status kept_counts(const sparsed_select_params* sp, int nb, int* pb, int
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Whether the switch step can select from the row statistics of its own full-attention pass.
+bool step_uses_stats(const sparsed_shape* shape, const sparsed_select_params* params) {
+  return params->block_size != 32 && shape->seq_len <= 131072;
+}
+
 // Checks the caller's pattern buffers against the number of rows and kept blocks per row and
 // fills in the host-side fields of `out`.
 sparsed_status prepare_pattern(sparsed_pattern* out, int batch, int heads_q, int nb, int block_size, int k_total) {
@@ -259,6 +264,24 @@ sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape* shape, c
       if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
       *out_bytes = SPARSED_STATUS_BYTES +
                    pooled_qk_means_bytes(shape->batch, shape->heads_q, shape->heads_kv, shape->seq_len / params->block_size);
+      return SPARSED_OK;
+    }
+    case SPARSED_OP_ATTENTION_STEP: {
+      if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
+      if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+      if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
+      if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
+      const size_t nb = static_cast<size_t>(shape->seq_len / params->block_size);
+      const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
+      const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
+      if (step_uses_stats(shape, params)) {
+        size_t stats = 0;
+        sparsed_status st = sparsed_tile_stats_bytes(shape, &stats);
+        if (st != SPARSED_OK) return st;
+        *out_bytes = SPARSED_STATUS_BYTES + lse_bytes + stats;
+      } else {
+        *out_bytes = SPARSED_STATUS_BYTES + round_up(bh * nb * nb * 4, 256) + lse_bytes;
+      }
       return SPARSED_OK;
     }
     default:
@@ -520,6 +543,39 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   if (e != cudaSuccess) return cuda_fail(e);
   if (fused) return SPARSED_OK;
   return run_topk(scores, shape->batch, shape->heads_q, nb, params->block_size, pb, k_pre, k_gen, out, stream);
+}
+
+sparsed_status sparsed_attention_step(const sparsed_shape* shape, const sparsed_select_params* params,
+                                      int32_t step_1based, int32_t total_steps, double skip, const void* q,
+                                      const void* k, const void* v, void* o, sparsed_pattern* pattern, void* ws,
+                                      size_t ws_bytes, void* cuda_stream, int32_t* mode_out_or_null) {
+  const int32_t mode = sparsed_schedule_mode(step_1based, total_steps, skip);
+  if (mode < 0) return SPARSED_ERR_INVALID_ARG;
+  if (mode_out_or_null != nullptr) *mode_out_or_null = mode;
+  if (mode == SPARSED_MODE_FULL) return sparsed_attn_full(shape, q, k, v, o, nullptr, ws, ws_bytes, cuda_stream);
+  if (mode == SPARSED_MODE_SPARSE) return sparsed_attn_sparse(shape, pattern, q, k, v, o, ws, ws_bytes, cuda_stream);
+  // the switch step
+  if (shape == nullptr || params == nullptr) return SPARSED_ERR_INVALID_ARG;
+  size_t need = 0;
+  sparsed_status st = sparsed_workspace_bytes(SPARSED_OP_ATTENTION_STEP, shape, params, &need);
+  if (st != SPARSED_OK) return st;
+  if (ws == nullptr || ws_bytes < need) return SPARSED_ERR_WORKSPACE;
+  const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
+  const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  if (step_uses_stats(shape, params)) {
+    float* lse = reinterpret_cast<float*>(base + SPARSED_STATUS_BYTES);
+    float* stats = reinterpret_cast<float*>(base + SPARSED_STATUS_BYTES + lse_bytes);
+    if ((st = sparsed_attn_full_stats(shape, q, k, v, o, lse, stats, ws, ws_bytes, cuda_stream)) != SPARSED_OK) return st;
+    return sparsed_select_from_stats(shape, params, lse, stats, pattern, nullptr, ws, ws_bytes, cuda_stream);
+  }
+  // [status][A' scratch of sparsed_select_pattern][LSE of the full pass]
+  const size_t nb = static_cast<size_t>(shape->seq_len / params->block_size);
+  const size_t score_bytes = round_up(bh * nb * nb * 4, 256);
+  float* lse = reinterpret_cast<float*>(base + SPARSED_STATUS_BYTES + score_bytes);
+  if ((st = sparsed_attn_full(shape, q, k, v, o, lse, ws, ws_bytes, cuda_stream)) != SPARSED_OK) return st;
+  return sparsed_select_pattern(shape, params, q, k, lse, pattern, nullptr, ws, SPARSED_STATUS_BYTES + score_bytes,
+                                cuda_stream);
 }
 
 sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int32_t num_blocks, int32_t block_size,

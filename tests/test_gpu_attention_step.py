@@ -1,0 +1,82 @@
+"""Algorithm 1 through the single-call entry point: every step of a short denoising schedule on the GPU
+against the oracle's step-by-step composition, on inputs that change from step to step; both ways the
+switch step can select (row statistics of its own pass; the two-pass scorer for 32-token blocks)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_24014_b200 as sd
+from oracle import sparsed_oracle as orc
+from paper_2509_24014_b200 import synthetic as syn
+from tests.parity_util import check_outputs, to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("bs,L,rho,prefill,T,skip", [
+    (64, 1024, 0.3, 0, 5, 0.4),        # switch at step 2, selection from the full pass's statistics
+    (128, 1536, 0.25, 512, 4, 0.5),    # isolated regions, switch at step 2
+    (32, 512, 0.5, 128, 4, 0.25),      # 32-token blocks: the switch step falls back to the two-pass scorer
+    (64, 768, 0.3, 0, 3, 0.0),         # skip = 0: the first step is the switch step
+])
+def test_schedule_through_one_entry_point(bs, L, rho, prefill, T, skip):
+    cfg = syn.AttnConfig("step", 1, 4, 2, L, 128, bs, rho, prefill, seed=900 + bs, total_steps=T, skip=skip,
+                         step_noise=0.05)
+    base = syn.make_base(cfg, DEV)
+    nb = L // bs
+    params = sd.make_params(bs, rho, prefill)
+    kp, kg = sd.sparsed_kept_per_row(params, L)
+    pat, rp_t, ci_t = sd.new_pattern(1, 4, nb, kp + kg, DEV)
+    q0, k0, _ = syn.make_qkv(cfg, DEV, step=1, base=base)
+    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_ATTENTION_STEP, sd.make_shape(q0, k0), params), DEV)
+    s_switch = orc.switch_step(T, skip)
+    pattern_ref = None
+    modes = []
+    for step in range(1, T + 1):
+        q, k, v = syn.make_qkv(cfg, DEV, step=step, base=base)
+        o = torch.empty_like(q)
+        # only the switch step needs the large workspace
+        ws_step = ws if step == s_switch else ws[: sd.sparsed_workspace_bytes(sd.OP_ATTN_FULL)]
+        mode = sd.sparsed_attention_step(q, k, v, o, params, step, T, skip, pat, ws_step)
+        torch.cuda.synchronize()
+        modes.append(mode)
+        assert mode == orc.schedule_mode(step, T, skip)
+        qd, kd, vd = to_f64(q), to_f64(k), to_f64(v)
+        if step <= s_switch:
+            o_ref = orc.sparsed_attention(qd, kd, vd, step, T, rho, skip, bs, prefill)[0]
+            check_outputs(o, o_ref, f"step {step} (full)")
+            if step == s_switch:
+                # the GPU's pattern: valid, the right counts, and the oracle's wherever the ranking is clear
+                rp, ci = rp_t.cpu().numpy(), ci_t.cpu().numpy()
+                a_ref = orc.pooled_scores(qd, kd, bs)
+                rp64, ci64 = orc.select_blocks(a_ref, bs, prefill, rho)
+                np.testing.assert_array_equal(rp, rp64)
+                same = sum(list(ci[rp[r]:rp[r + 1]]) == list(ci64[rp64[r]:rp64[r + 1]]) for r in range(4 * nb))
+                assert same >= 0.5 * 4 * nb, same
+                pattern_ref = (rp, ci)
+        else:
+            o_ref, _ = orc.sparsed_attention(qd, kd, vd, step, T, rho, skip, bs, prefill, pattern=pattern_ref)
+            check_outputs(o, o_ref, f"step {step} (sparse)")
+    assert modes == [sd.MODE_FULL] * (s_switch - 1) + [sd.MODE_FULL_AND_SELECT] + [sd.MODE_SPARSE] * (T - s_switch)
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+
+
+def test_step_argument_checks():
+    cfg = syn.AttnConfig("step", 1, 1, 1, 256, 128, 128, 0.5, 0, seed=1)
+    q, k, v = syn.make_qkv(cfg, DEV)
+    o = torch.empty_like(q)
+    params = sd.make_params(128, 0.5, 0)
+    pat, _, _ = sd.new_pattern(1, 1, 2, 1, DEV)
+    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_ATTENTION_STEP, sd.make_shape(q, k), params), DEV)
+    for bad_step, T, skip in ((0, 4, 0.5), (5, 4, 0.5), (1, 4, 1.5)):
+        with pytest.raises(sd.SparsedError) as e:
+            sd.sparsed_attention_step(q, k, v, o, params, bad_step, T, skip, pat, ws)
+        assert e.value.status == 1
+    with pytest.raises(sd.SparsedError) as e:     # the switch step with a status-only workspace
+        sd.sparsed_attention_step(q, k, v, o, params, 2, 4, 0.5, pat, ws[:256])
+    assert e.value.status == 4
+    assert sd.sparsed_attention_step(q, k, v, o, params, 2, 4, 0.5, pat, ws) == sd.MODE_FULL_AND_SELECT
+    assert sd.sparsed_attention_step(q, k, v, o, params, 3, 4, 0.5, pat, ws[:256]) == sd.MODE_SPARSE
+    torch.cuda.synchronize()
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
