@@ -129,7 +129,8 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
  *   sparsed_attn_full_stats   = sparsed_attn_full that also records, for every query row and
  *                               every 64-key tile, log2 of the tile's share of the row's softmax
  *                               denominator (tile_stats, device fp32, sparsed_tile_stats_bytes()
- *                               bytes, layout [batch*heads_q][ceil(seq_len/64)][seq_len]);
+ *                               bytes, layout [batch*heads_q][ceil(seq_len/128)][ceil(seq_len/64)][128]:
+ *                               128-row query tile, 64-key tile, row in the query tile);
  *                               lse is required here.
  *   sparsed_select_from_stats = pools those statistics into A' (2^(stat - LSE) is the
  *                               probability mass a row puts on a tile), ranks it as
@@ -202,7 +203,7 @@ int32_t sparsed_switch_step(int32_t total_steps, double skip);
  * sparsed_select_pattern, written at the switch step and only read afterwards; the caller keeps it
  * (one per layer) across steps. ws: device workspace, zeroed status block first; the switch step
  * needs sparsed_workspace_bytes(SPARSED_OP_ATTENTION_STEP, shape, params) bytes (row statistics of
- * the full pass: 4 * seq_len * ceil(seq_len / 64) bytes per head), every other step only
+ * the full pass: about 4 * seq_len * ceil(seq_len / 64) bytes per head), every other step only
  * SPARSED_STATUS_BYTES. mode_out_or_null (host) receives the mode that ran. Errors as for the calls
  * it makes; INVALID_ARG for a step outside 1..total_steps or skip outside [0, 1]. Asynchronous.
  */

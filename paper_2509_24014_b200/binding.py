@@ -245,9 +245,9 @@ def sparsed_tile_stats_bytes(shape: Shape) -> int:
 
 
 def new_tile_stats(q: torch.Tensor) -> torch.Tensor:
-    """Caller-owned buffer for sparsed_attn_full_stats: fp32 [B*Hq, ceil(L/64), L]."""
+    """Caller-owned buffer for sparsed_attn_full_stats: fp32 [B*Hq, ceil(L/128), ceil(L/64), 128]."""
     B, Hq, L, _ = q.shape
-    return torch.empty(B * Hq, (L + 63) // 64, L, dtype=torch.float32, device=q.device)
+    return torch.empty(B * Hq, (L + 127) // 128, (L + 63) // 64, 128, dtype=torch.float32, device=q.device)
 
 
 def sparsed_attn_full_stats(q, k, v, o, lse: torch.Tensor, tile_stats: torch.Tensor, ws: torch.Tensor,

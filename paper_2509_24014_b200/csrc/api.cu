@@ -337,7 +337,8 @@ sparsed_status sparsed_tile_stats_bytes(const sparsed_shape* shape, size_t* out_
   if (shape == nullptr || out_bytes == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
   const size_t tiles = (static_cast<size_t>(shape->seq_len) + 63) / 64;
-  *out_bytes = static_cast<size_t>(shape->batch) * shape->heads_q * tiles * static_cast<size_t>(shape->seq_len) * 4;
+  const size_t q_tiles = (static_cast<size_t>(shape->seq_len) + 127) / 128;
+  *out_bytes = static_cast<size_t>(shape->batch) * shape->heads_q * q_tiles * tiles * 128 * 4;
   return SPARSED_OK;
 }
 

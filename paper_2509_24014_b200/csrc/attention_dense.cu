@@ -16,7 +16,9 @@
 // The streams share nothing else (own S buffers, O accumulator, maxima), so they drift apart and
 // one stream's softmax overlaps the other's MMAs. Tensor memory: 2 x (2 x 64 S + 128 O) = 512
 // columns; shared memory 208 KB. Optional outputs: LSE, and the per-(row, 64-key tile) statistic
-// m + log2(sum p) from which the switch step's pooled scores are formed.
+// m + log2(sum p) from which the switch step's pooled scores are formed (laid out
+// [batch*head][128-row query tile][key tile][row], so that both this kernel's writes and the
+// pooling kernel's reads are contiguous per query tile).
 #include "internal.h"
 
 namespace sparsed {
@@ -285,9 +287,10 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
         l += sum;
         if (p.tile_lse != nullptr) {
-          const int row_g = q_row0 + row_t;
-          if (row_g < p.seq_len)
-            __stcs(p.tile_lse + (static_cast<int64_t>(bh) * num_tiles + t) * p.seq_len + row_g, m_used + __log2f(sum));
+          // [bh][query tile][key tile][row in tile]: a stream's writes are consecutive 512-byte pieces
+          const int64_t qt = static_cast<int64_t>(bh) * p.num_q_tiles + (2 * pair + s);
+          if (q_row0 + row_t < p.seq_len)
+            __stcs(p.tile_lse + (qt * num_tiles + t) * kTileM + row_t, m_used + __log2f(sum));
         }
         tmem_st32(tS, pk);
         tmem_wait_st();

@@ -14,7 +14,7 @@ struct AttnParams {
   void* o;                 // bf16 [B,Hq,L,D]
   int64_t o_stride_b, o_stride_h, o_stride_t;
   float* lse;              // fp32 [B,Hq,L] or null
-  float* tile_lse;         // fp32 [B*Hq, ceil(L/64), L] or null: base-2 log-sum-exp of each row over each 64-key tile
+  float* tile_lse;         // fp32 [B*Hq, ceil(L/128), ceil(L/64), 128] or null: base-2 log-sum-exp of each row over each 64-key tile
   int seq_len;
   int heads_q;
   int group;               // heads_q / heads_kv
@@ -46,7 +46,7 @@ constexpr int kFusedTopkMaxBlocks = 1024;
 
 // Parameters of the kernel that pools per-tile row statistics into A' and ranks it.
 struct PoolParams {
-  const float* tile_lse;   // fp32 [B*Hq, tiles, L], base-2
+  const float* tile_lse;   // fp32 [B*Hq, ceil(L/128), tiles, 128], base-2
   const float* lse;        // fp32 [B,Hq,L], natural log
   float* scores;           // fp32 [B,Hq,nb,nb] or null
   int32_t* row_ptr;

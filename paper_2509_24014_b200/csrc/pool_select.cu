@@ -9,12 +9,13 @@
 // of block jb, divided by block_size^2.
 //
 // One CTA owns one 128-row query tile of one (batch, head). Statistics are read with 16-byte
-// loads (four consecutive rows of one tile; row-fastest layout), sixteen in flight per thread,
+// loads (four consecutive rows of one tile; the layout [bh][128-row query tile][key tile][row]
+// makes a CTA's reads one contiguous run), sixteen in flight per thread,
 // exponentiated, parked in shared memory in chunks of 64 tiles, and summed per tile and row half
 // in a fixed, bank-conflict-free order (bitwise reproducible).
 // The CTA then holds its block-row(s) of A' in shared memory, optionally writes them out, and
 // warp 0 ranks them (warp_select_row) and writes the CSR lists. HBM-bound:
-// 4 * L * ceil(L/64) bytes read per (batch, head).
+// 4 * 128 * ceil(L/128) * ceil(L/64) bytes read per (batch, head).
 #include "internal.h"
 #include "topk_device.cuh"
 
@@ -76,7 +77,8 @@ __global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams 
     const float c = 1.44269504088896341f;
     lse2 = make_float4(t.x * c, t.y * c, t.z * c, t.w * c);
   }
-  const float* src = p.tile_lse + static_cast<int64_t>(bh) * n_tiles * L + row4;
+  // statistics layout [bh][query tile][key tile][128 rows]: this CTA's share is one contiguous run
+  const float* src = p.tile_lse + (static_cast<int64_t>(bh) * num_q_tiles + q_tile) * n_tiles * kRows + lane * 4;
 
   for (int c0 = 0; c0 < n_tiles; c0 += kChunk) {
     const int n_here = min(kChunk, n_tiles - c0);
@@ -86,7 +88,7 @@ __global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams 
       for (int u = 0; u < kInFlight; ++u) {
         const int t = tt + 4 * u;
         v[u] = (rows_valid && t < n_here)
-                   ? __ldcs(reinterpret_cast<const float4*>(src + static_cast<int64_t>(c0 + t) * L))
+                   ? __ldcs(reinterpret_cast<const float4*>(src + static_cast<int64_t>(c0 + t) * kRows))
                    : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
       }
 #pragma unroll
