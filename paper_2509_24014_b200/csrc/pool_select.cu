@@ -10,9 +10,10 @@
 //
 // One CTA owns one 128-row query tile of one (batch, head). Statistics are read with 16-byte
 // loads (four consecutive rows of one tile; the layout [bh][128-row query tile][key tile][row]
-// makes a CTA's reads one contiguous run), sixteen in flight per thread,
-// exponentiated, parked in shared memory in chunks of 64 tiles, and summed per tile and row half
-// in a fixed, bank-conflict-free order (bitwise reproducible).
+// makes a CTA's reads one contiguous run), eight in flight per thread and six CTAs per SM (the
+// best point of a sweep: 5.9 TB/s at 64k), exponentiated, parked in shared memory in chunks of 32
+// tiles, and summed per tile and row half in a fixed, bank-conflict-free order (bitwise
+// reproducible); the next chunk's loads are issued before the current chunk is summed.
 // The CTA then holds its block-row(s) of A' in shared memory, optionally writes them out, and
 // warp 0 ranks them (warp_select_row) and writes the CSR lists. HBM-bound:
 // 4 * 128 * ceil(L/128) * ceil(L/64) bytes read per (batch, head).
@@ -23,12 +24,15 @@ namespace sparsed {
 namespace {
 
 constexpr int kRows = 128;
-constexpr int kChunk = 64;          // tiles per transposition chunk
-constexpr int kPitch = kRows + 4;   // floats per chunk row: keeps float4 stores aligned
 #ifndef SPARSED_POOL_IN_FLIGHT
-#define SPARSED_POOL_IN_FLIGHT 16
+#define SPARSED_POOL_IN_FLIGHT 8
+#endif
+#ifndef SPARSED_POOL_CTAS_PER_SM
+#define SPARSED_POOL_CTAS_PER_SM 6
 #endif
 constexpr int kInFlight = SPARSED_POOL_IN_FLIGHT;  // 16-byte loads each thread keeps in flight
+constexpr int kChunk = 4 * kInFlight;  // tiles per transposition chunk: one batch of loads per thread
+constexpr int kPitch = kRows + 4;   // floats per chunk row: keeps float4 stores aligned
 constexpr int kMaxTiles = 2048;     // seq_len <= 131072
 
 // Shared memory (dynamic, sized for the actual sequence): the transposition chunk, the per-tile
@@ -45,7 +49,7 @@ __host__ __device__ inline size_t pool_smem_bytes(int n_tiles, int nb) {
          sizeof(int) * 256;
 }
 
-__global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams p) {
+__global__ void __launch_bounds__(kRows, SPARSED_POOL_CTAS_PER_SM) pool_select_kernel(const PoolParams p) {
   extern __shared__ __align__(16) uint8_t pool_smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int L = p.seq_len;
@@ -80,34 +84,41 @@ __global__ void __launch_bounds__(kRows, 4) pool_select_kernel(const PoolParams 
   // statistics layout [bh][query tile][key tile][128 rows]: this CTA's share is one contiguous run
   const float* src = p.tile_lse + (static_cast<int64_t>(bh) * num_q_tiles + q_tile) * n_tiles * kRows + lane * 4;
 
+  // One batch = this thread's kInFlight loads of a chunk (warp w takes tiles w, w+4, ... of it). The
+  // next chunk's batch is issued before the current chunk is summed, so loads stay in flight
+  // through the shared-memory phase.
+  static_assert(kChunk == 4 * kInFlight, "one batch of loads per thread covers one chunk");
+  float4 v[kInFlight];
+  auto issue = [&](int c0) {
+    const int n_here = min(kChunk, n_tiles - c0);
+#pragma unroll
+    for (int u = 0; u < kInFlight; ++u) {
+      const int t = warp + 4 * u;
+      v[u] = (rows_valid && t < n_here)
+                 ? __ldcs(reinterpret_cast<const float4*>(src + static_cast<int64_t>(c0 + t) * kRows))
+                 : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+  };
+  issue(0);
   for (int c0 = 0; c0 < n_tiles; c0 += kChunk) {
     const int n_here = min(kChunk, n_tiles - c0);
-    for (int tt = warp; tt < n_here; tt += 4 * kInFlight) {
-      float4 v[kInFlight];
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) {
-        const int t = tt + 4 * u;
-        v[u] = (rows_valid && t < n_here)
-                   ? __ldcs(reinterpret_cast<const float4*>(src + static_cast<int64_t>(c0 + t) * kRows))
-                   : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-      }
-#pragma unroll
-      for (int u = 0; u < kInFlight; ++u) {
-        const int t = tt + 4 * u;
-        if (t < n_here) {
-          const float4 e = make_float4(fast_exp2(v[u].x - lse2.x), fast_exp2(v[u].y - lse2.y),
-                                       fast_exp2(v[u].z - lse2.z), fast_exp2(v[u].w - lse2.w));
-          *reinterpret_cast<float4*>(sm.chunk + t * kPitch + lane * 4) = e;
-        }
+    for (int u = 0; u < kInFlight; ++u) {
+      const int t = warp + 4 * u;
+      if (t < n_here) {
+        const float4 e = make_float4(fast_exp2(v[u].x - lse2.x), fast_exp2(v[u].y - lse2.y),
+                                     fast_exp2(v[u].z - lse2.z), fast_exp2(v[u].w - lse2.w));
+        *reinterpret_cast<float4*>(sm.chunk + t * kPitch + lane * 4) = e;
       }
     }
     __syncthreads();
+    if (c0 + kChunk < n_tiles) issue(c0 + kChunk);
     {
       // Summing: thread j < 64 adds rows 0-63 of tile j, thread j + 64 rows 64-127. Each thread
       // starts at its own rotation of the 64 rows so that a warp's reads hit 32 different banks;
       // the order is fixed per tile, so the result is reproducible.
-      const int j = tid & 63, half = tid >> 6;
-      if (j < n_here) {
+      const int half = tid >> 6;
+      for (int j = tid & 63; j < n_here; j += 64) {
         const float* rowp = sm.chunk + j * kPitch + half * 64;
         float acc = 0.f;
 #pragma unroll 8
