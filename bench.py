@@ -41,13 +41,13 @@ METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at
 # summarised under profiles/; keyed by (kernel, workload). None where no capture exists.
 NCU_DRAM_TRAFFIC = {
     # profiles/ncu_dram_bytes_c4_step_kernels.md (1-pass capture on the full-size workload)
-    ("attn_dense_pair_kernel", "c4"): 1890352128 + 9088306944,
-    ("pool_select_kernel", "c4"): 8598400256 + 39179008,
-    ("attn_kernel<sparse>", "c4"): 1257575936 + 515790592,
+    ("attn_dense_pair_kernel", "c4"): 1853606144 + 9088952832,
+    ("pool_select_kernel", "c4"): 8598426368 + 41508096,
+    ("attn_kernel<sparse>", "c4"): 1250340864 + 516116992,
     # profiles/ncu_full_c2_all_kernels.md, profiles/ncu_full_topk_c4.md
-    ("attn_dense_pair_kernel", "c2"): 201678336 + 160317440,
-    ("pool_select_kernel", "c2"): 135333376 + 3458048,
-    ("attn_kernel<sparse>", "c2"): 156412416 + 42705920,
+    ("attn_dense_pair_kernel", "c2"): 201481728 + 158934272,
+    ("pool_select_kernel", "c2"): 135332352 + 3845632,
+    ("attn_kernel<sparse>", "c2"): 156542720 + 41992192,
     ("topk_csr_kernel", "c4"): 33585920,
 }
 
