@@ -129,3 +129,53 @@ def test_batched_long_context_settings(batch, seq_len, gen_len):
         kept = ci[rp[r]:rp[r + 1]]
         check_outputs(o_sp[b, h, rows], orc.head_sparse_rows(qh, kh, vh, ib, kept, bs),
                       f"batched sparse b{b} h{h} ib{ib}")
+
+
+def test_token_major_layout_through_every_entry_point():
+    """Q, K, V and O as [batch, token, head, dim] (what a fused QKV projection writes), passed by strides:
+    full + statistics, both selections, the block-mean estimate and sparse attention."""
+    B, L, Hq, Hkv, bs, rho, prefill = 2, 640, 4, 2, 64, 0.3, 128
+    cfg = syn.AttnConfig("tm", B, Hq, Hkv, L, 128, bs, rho, prefill, seed=123)
+    qc, kc, vc = syn.make_qkv(cfg, DEV)
+    q = qc.transpose(1, 2).contiguous().transpose(1, 2)     # same values, token-major memory
+    k = kc.transpose(1, 2).contiguous().transpose(1, 2)
+    v = vc.transpose(1, 2).contiguous().transpose(1, 2)
+    assert not q.is_contiguous() and q.stride(2) == Hq * 128
+    o = torch.empty(B, L, Hq, 128, dtype=torch.bfloat16, device=DEV).transpose(1, 2)
+    nb = L // bs
+    ws = sd.new_workspace(1 << 22, DEV)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=DEV)
+    stats = sd.new_tile_stats(q)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+    qd, kd, vd = to_f64(q), to_f64(k), to_f64(v)
+    o_ref, lse_ref = orc.attn_full(qd, kd, vd)
+    check_outputs(o, o_ref, "token-major full")
+    np.testing.assert_allclose(to_f64(lse), lse_ref, atol=3e-5, rtol=3e-6)
+    params = sd.make_params(bs, rho, prefill)
+    kp, kg = sd.sparsed_kept_per_row(params, L)
+    a_ref = orc.pooled_scores(qd, kd, bs)
+    lists = []
+    for path in ("stats", "two_pass"):
+        pat, rp_t, ci_t = sd.new_pattern(B, Hq, nb, kp + kg, DEV)
+        scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=DEV)
+        if path == "stats":
+            sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws, scores_out=scores)
+        else:
+            sd.sparsed_select_pattern(q, k, params, pat, ws, scores_out=scores)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(scores.cpu().numpy(), a_ref, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+        rp, ci = orc.select_blocks(scores.cpu().numpy(), bs, prefill, rho)
+        np.testing.assert_array_equal(ci_t.cpu().numpy(), ci)
+        lists.append((pat, rp, ci, rp_t, ci_t))
+    pat_e, rp_e, ci_e = sd.new_pattern(B, Hq, nb, kp + kg, DEV)
+    est = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=DEV)
+    ws_e = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_POOLED_QK, sd.make_shape(q, k), params), DEV)
+    sd.sparsed_select_pattern_pooled_qk(q, k, params, pat_e, ws_e, scores_out=est)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(est.cpu().numpy(), orc.pooled_qk_scores(qd, kd, bs), rtol=5e-5, atol=1e-12)
+    pat, rp, ci, _, _ = lists[0]
+    o_sp = torch.empty(B, L, Hq, 128, dtype=torch.bfloat16, device=DEV).transpose(1, 2)
+    sd.sparsed_attn_sparse(q, k, v, o_sp, pat, ws)
+    torch.cuda.synchronize()
+    check_outputs(o_sp, orc.attn_sparse(qd, kd, vd, rp, ci, bs), "token-major sparse")
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
