@@ -70,14 +70,19 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index = index
-        self.lines = []
+        self.lines = []      # (arrival time, text)
         self.proc = None
+        self.t_begin = 0.0
+
+    def mark_begin(self):
+        """Samples that arrive before this moment (warm-up) are not counted."""
+        self.t_begin = time.monotonic()
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -85,7 +90,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
 
     def stop(self):
         if self.proc is None:
@@ -97,7 +102,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for t_line, ln in self.lines:
+            if t_line < self.t_begin:
+                continue
             parts = [x.strip() for x in ln.split(",")]
             if len(parts) < 8:
                 continue
@@ -308,15 +315,16 @@ def run_ours(args, cfg):
         if events is not None:
             events.append(marks)
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()          # nvidia-smi needs a moment to start streaming: launch it before the warm-up
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
+    sampler.mark_begin()
     events = []
     t_begin, t_end = ev(), ev()
     t_begin.record()
