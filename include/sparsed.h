@@ -14,6 +14,9 @@
  *    [batch, heads_kv, seq_len, head_dim], bf16, head_dim contiguous. Strides for
  *    (batch, head, token) are given in elements; all-zero strides mean "contiguous".
  *    Base pointers must be 16-byte aligned and every stride a multiple of 8 elements.
+ *    The fp32 side buffers (lse, tile_stats, scores, scores_out) and the workspace must be
+ *    16-byte aligned too (the kernels read them with 16-byte loads), row_ptr and col_idx
+ *    4-byte aligned; anything else is refused with SPARSED_ERR_ALIGNMENT before any launch.
  *  - Grouped-query attention: query head h reads key/value head h / (heads_q / heads_kv).
  *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *    stream) and return without synchronising. Argument problems are detected on the
@@ -211,6 +214,28 @@ sparsed_status sparsed_attention_step(const sparsed_shape *shape, const sparsed_
                                       int32_t step_1based, int32_t total_steps, double skip, const void *q,
                                       const void *k, const void *v, void *o, sparsed_pattern *pattern, void *ws,
                                       size_t ws_bytes, void *cuda_stream, int32_t *mode_out_or_null);
+
+/*
+ * sparsed_attention_step with one of the method's components switched off: the rows of the paper's
+ * component ablation (Table 2) as modes of the same call, for timing and for comparison.
+ *   SPARSED_VARIANT_NO_REUSE     "- Sparse Reusing": every sparse step first selects its own pattern from
+ *                                that step's Q and K (sparsed_select_pattern with no LSE: a row-statistics
+ *                                pass, pooled scoring, ranking) and then attends on it; `pattern` is
+ *                                overwritten at every sparse step. Such steps need
+ *                                sparsed_workspace_bytes(SPARSED_OP_SELECT_PATTERN, ...) bytes of workspace.
+ *   SPARSED_VARIANT_NO_ISOLATION "- Isolated Selection": prefill_len is ignored, one top-rho% over all key
+ *                                blocks (Eq. 5 without the split of Eq. 6).
+ * ("- Skipping Sparse" is skip = 0: the first step is the switch step.) Flags may be combined; 0 is
+ * sparsed_attention_step itself. Everything else as for sparsed_attention_step; INVALID_ARG for
+ * unknown flag bits.
+ */
+#define SPARSED_VARIANT_NO_REUSE 1
+#define SPARSED_VARIANT_NO_ISOLATION 2
+sparsed_status sparsed_attention_step_variant(const sparsed_shape *shape, const sparsed_select_params *params,
+                                              int32_t variant, int32_t step_1based, int32_t total_steps,
+                                              double skip, const void *q, const void *k, const void *v, void *o,
+                                              sparsed_pattern *pattern, void *ws, size_t ws_bytes,
+                                              void *cuda_stream, int32_t *mode_out_or_null);
 
 /*
  * Number of key blocks kept per query block in the prefill and generation regions

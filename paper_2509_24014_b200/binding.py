@@ -18,6 +18,7 @@ STATUS_BYTES = 256
 (OP_ATTN_FULL, OP_SELECT_PATTERN, OP_SELECT_FROM_SCORES, OP_ATTN_SPARSE, OP_PATTERN_VALIDATE, OP_SELECT_POOLED_QK,
  OP_ATTENTION_STEP) = range(7)
 MODE_FULL, MODE_FULL_AND_SELECT, MODE_SPARSE = 0, 1, 2
+VARIANT_NO_REUSE, VARIANT_NO_ISOLATION = 1, 2
 
 EXPORTED_SYMBOLS = (
     "sparsed_attn_full", "sparsed_select_pattern", "sparsed_select_from_scores", "sparsed_attn_sparse",
@@ -26,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "sparsed_status_string", "sparsed_last_cuda_error", "sparsed_select_pattern_static",
     "sparsed_tile_stats_bytes", "sparsed_attn_full_stats", "sparsed_select_from_stats",
     "sparsed_build_window_pattern", "sparsed_selftest_wait_timeout", "sparsed_select_pattern_pooled_qk",
-    "sparsed_attention_step",
+    "sparsed_attention_step", "sparsed_attention_step_variant",
 )
 
 
@@ -80,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.sparsed_select_pattern_pooled_qk.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_attention_step.argtypes = [P(Shape), P(SelectParams), i32, i32, ctypes.c_double, vp, vp, vp, vp,
                                            P(Pattern), vp, sz, vp, P(i32)]
+    lib.sparsed_attention_step_variant.argtypes = [P(Shape), P(SelectParams), i32, i32, i32, ctypes.c_double, vp, vp, vp,
+                                                   vp, P(Pattern), vp, sz, vp, P(i32)]
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
     lib.sparsed_build_window_pattern.argtypes = [i32, i32, i32, i32, i32, i32, P(Pattern), vp]
     lib.sparsed_selftest_wait_timeout.argtypes = [vp, sz, vp]
@@ -235,6 +238,19 @@ def sparsed_attention_step(q, k, v, o, params: SelectParams, step_1based: int, t
         ctypes.byref(shape), ctypes.byref(params), int(step_1based), int(total_steps), float(skip), q.data_ptr(),
         k.data_ptr(), v.data_ptr(), o.data_ptr(), ctypes.byref(pattern), ws.data_ptr(), ws.numel(), _stream(q),
         ctypes.byref(mode)), "sparsed_attention_step")
+    return int(mode.value)
+
+
+def sparsed_attention_step_variant(q, k, v, o, params: SelectParams, variant: int, step_1based: int,
+                                   total_steps: int, skip: float, pattern: Pattern, ws: torch.Tensor,
+                                   softmax_scale: float = 0.0, shape: Optional[Shape] = None) -> int:
+    """sparsed_attention_step with components of the method switched off (VARIANT_* flags)."""
+    shape = shape or make_shape(q, k, v, o, softmax_scale)
+    mode = ctypes.c_int32(-1)
+    _check(load_library().sparsed_attention_step_variant(
+        ctypes.byref(shape), ctypes.byref(params), int(variant), int(step_1based), int(total_steps), float(skip),
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), ctypes.byref(pattern), ws.data_ptr(), ws.numel(),
+        _stream(q), ctypes.byref(mode)), "sparsed_attention_step_variant")
     return int(mode.value)
 
 

@@ -1,16 +1,26 @@
-"""Builds the C-ABI shared library (libsparsed.so) in-tree with nvcc for sm_100a."""
+"""Builds the C-ABI shared library (libsparsed.so) in-tree with nvcc for sm_100a.
+
+Each .cu file is compiled to an object of its own (in parallel, skipped when the object is newer
+than the source and every header), then the objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import os
 import shutil
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
+OBJ_DIR = os.path.join(PKG_DIR, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libsparsed.so")
-SOURCES = ["api.cu", "attention.cu", "attention_dense.cu", "scoring.cu", "topk.cu", "pool_select.cu", "patterns.cu", "pooled_qk.cu"]
-HEADERS = ["internal.h", "sm100_primitives.cuh", "topk_device.cuh", os.path.join("..", "..", "include", "sparsed.h")]
+SOURCES = ["api.cu", "attention.cu", "attention_dense.cu", "scoring.cu", "topk.cu", "pool_select.cu", "patterns.cu",
+           "pooled_qk.cu"]
+HEADERS = ["internal.h", "sm100_primitives.cuh", "softmax_pipeline.cuh", "topk_device.cuh",
+           os.path.join("..", "..", "include", "sparsed.h")]
+ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
+COMMON_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC"]
 
 
 def _nvcc() -> str:
@@ -20,28 +30,50 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found; the SparseD library needs the CUDA 12.9 toolkit to build")
 
 
+def _deps():
+    return [os.path.join(CSRC, s) for s in SOURCES + HEADERS if os.path.exists(os.path.join(CSRC, s))]
+
+
 def is_stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = [os.path.join(CSRC, s) for s in SOURCES + HEADERS]
-    return any(os.path.getmtime(d) > t for d in deps)
+    return any(os.path.getmtime(d) > t for d in _deps())
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and not is_stale():
-        return LIB_PATH
-    tmp_path = f"{LIB_PATH}.tmp{os.getpid()}.so"
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "-shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v" if verbose else "-O3",
-           "-o", tmp_path] + [os.path.join(CSRC, s) for s in SOURCES]
+def _compile_one(nvcc: str, src: str, obj: str, verbose: bool, extra):
+    cmd = [nvcc] + ARCH_FLAGS + COMMON_FLAGS + list(extra) + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose:
-        sys.stderr.write(res.stderr)
+    return src, res
+
+
+def build_library(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
+    if not force and not is_stale() and not extra_flags:
+        return LIB_PATH
+    nvcc = _nvcc()
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    header_time = max(os.path.getmtime(os.path.join(CSRC, h)) for h in HEADERS if os.path.exists(os.path.join(CSRC, h)))
+    jobs, objs = [], []
+    for s in SOURCES:
+        src = os.path.join(CSRC, s)
+        obj = os.path.join(OBJ_DIR, s.replace(".cu", ".o"))
+        objs.append(obj)
+        fresh = (os.path.exists(obj) and os.path.getmtime(obj) > max(os.path.getmtime(src), header_time))
+        if force or verbose or extra_flags or not fresh:
+            jobs.append((src, obj))
+    with ThreadPoolExecutor(max_workers=min(8, max(1, len(jobs)))) as pool:
+        results = list(pool.map(lambda j: _compile_one(nvcc, j[0], j[1], verbose, extra_flags), jobs))
+    for src, res in results:
+        if verbose:
+            sys.stderr.write(res.stderr)
+        if res.returncode != 0:
+            raise RuntimeError(f"nvcc failed on {src}:\n" + res.stdout + res.stderr)
+    tmp_path = f"{LIB_PATH}.tmp{os.getpid()}.so"
+    res = subprocess.run([nvcc] + ARCH_FLAGS + ["-shared", "-o", tmp_path] + objs, capture_output=True, text=True)
     if res.returncode != 0:
         if os.path.exists(tmp_path):
             os.remove(tmp_path)
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     os.replace(tmp_path, LIB_PATH)   # atomic: a concurrent loader never sees a half-written library
     return LIB_PATH
 

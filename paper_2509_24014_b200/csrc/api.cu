@@ -1,5 +1,6 @@
 // C ABI of the SparseD attention library: argument validation, tensor-map construction,
 // workspace layout and kernel dispatch. Declarations and contracts are in sparsed.h.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -37,9 +38,44 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// Host-side cache of encoded tensor maps. A map depends only on (base pointer, extents, strides,
+// box), not on the tensor's contents, so a denoising loop that calls with the same buffers every
+// step encodes each map once. Per thread (no locking), direct-mapped, 32 entries.
+struct TensorMapKey {
+  const void* base;
+  int64_t strides[3];
+  int32_t batch, heads, seq_len, box_rows;
+  bool operator==(const TensorMapKey& o) const {
+    return base == o.base && strides[0] == o.strides[0] && strides[1] == o.strides[1] && strides[2] == o.strides[2] &&
+           batch == o.batch && heads == o.heads && seq_len == o.seq_len && box_rows == o.box_rows;
+  }
+};
+struct TensorMapSlot {
+  TensorMapKey key;
+  CUtensorMap map;
+  bool valid;
+};
+constexpr int kTensorMapSlots = 32;
+thread_local TensorMapSlot g_tensor_maps[kTensorMapSlots] = {};
+
+uint32_t tensor_map_slot(const TensorMapKey& k) {
+  uint64_t h = reinterpret_cast<uintptr_t>(k.base) >> 4;
+  h = h * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(k.strides[1]);
+  h = h * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(k.strides[2]);
+  h = h * 0x9E3779B97F4A7C15ull + (static_cast<uint64_t>(k.seq_len) << 8 | static_cast<uint64_t>(k.box_rows));
+  h = h * 0x9E3779B97F4A7C15ull + (static_cast<uint64_t>(k.heads) << 16 | static_cast<uint64_t>(k.batch));
+  return static_cast<uint32_t>(h >> 40) % kTensorMapSlots;
+}
+
 // bf16 [B,H,L,128] tensor with element strides (batch, head, token); box = 64 x rows, 128B swizzle.
 sparsed_status make_tensor_map(CUtensorMap* out, const void* base, int batch, int heads, int seq_len,
                                const int64_t strides[3], int box_rows) {
+  TensorMapKey key{base, {strides[0], strides[1], strides[2]}, batch, heads, seq_len, box_rows};
+  TensorMapSlot& slot = g_tensor_maps[tensor_map_slot(key)];
+  if (slot.valid && slot.key == key) {
+    *out = slot.map;
+    return SPARSED_OK;
+  }
   EncodeTiledFn enc = encode_tiled_fn();
   if (enc == nullptr) return cuda_fail(cudaErrorNotSupported);
   cuuint64_t dims[4] = {128, static_cast<cuuint64_t>(seq_len), static_cast<cuuint64_t>(heads),
@@ -55,6 +91,9 @@ sparsed_status make_tensor_map(CUtensorMap* out, const void* base, int batch, in
     g_last_cuda_error = static_cast<int32_t>(r);
     return SPARSED_ERR_CUDA;
   }
+  slot.key = key;
+  slot.map = *out;
+  slot.valid = true;
   return SPARSED_OK;
 }
 
@@ -64,6 +103,13 @@ struct Resolved {
 };
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+// The workspace holds the status word (atomics) and fp32 arrays the kernels read with 16-byte loads.
+sparsed_status check_ws(const void* ws, size_t ws_bytes, size_t need) {
+  if (ws == nullptr || ws_bytes < need) return SPARSED_ERR_WORKSPACE;
+  return aligned16(ws) ? SPARSED_OK : SPARSED_ERR_ALIGNMENT;
+}
 
 void default_strides(const int64_t in[3], int heads, int seq_len, int64_t out[3]) {
   if (in[0] == 0 && in[1] == 0 && in[2] == 0) {
@@ -81,18 +127,12 @@ sparsed_status check_arch() {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e);
-  static int cached_major[64];
-  static bool cached[64] = {};
-  int major = 0;
-  if (dev >= 0 && dev < 64 && cached[dev]) {
-    major = cached_major[dev];
-  } else {
+  static std::atomic<int> cached_major[64];  // 0 = not looked up yet
+  int major = (dev >= 0 && dev < 64) ? cached_major[dev].load(std::memory_order_relaxed) : 0;
+  if (major == 0) {
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
     if (e != cudaSuccess) return cuda_fail(e);
-    if (dev >= 0 && dev < 64) {
-      cached_major[dev] = major;
-      cached[dev] = true;
-    }
+    if (dev >= 0 && dev < 64) cached_major[dev].store(major, std::memory_order_relaxed);
   }
   return major == 10 ? SPARSED_OK : SPARSED_ERR_ARCH;
 }
@@ -155,6 +195,7 @@ bool step_uses_stats(const sparsed_shape* shape, const sparsed_select_params* pa
 // fills in the host-side fields of `out`.
 sparsed_status prepare_pattern(sparsed_pattern* out, int batch, int heads_q, int nb, int block_size, int k_total) {
   if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if (!aligned4(out->row_ptr) || !aligned4(out->col_idx)) return SPARSED_ERR_ALIGNMENT;
   if (nb > 16384) return SPARSED_ERR_UNSUPPORTED;
   const int64_t rows = static_cast<int64_t>(batch) * heads_q * nb;
   const int64_t nnz = rows * k_total;
@@ -290,7 +331,8 @@ sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape* shape, c
 }
 
 sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  sparsed_status st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES);
+  if (st != SPARSED_OK) return st;
   cudaError_t e = cudaMemsetAsync(ws, 0, SPARSED_STATUS_BYTES, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
@@ -303,12 +345,14 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   if (st != SPARSED_OK) return st;
   if (q == nullptr || k == nullptr || v == nullptr || o == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SPARSED_ERR_ALIGNMENT;
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if (!aligned16(lse_or_null) || !aligned16(tile_lse_or_null)) return SPARSED_ERR_ALIGNMENT;
+  if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
+  const int kv_box_rows = 64;
   CUtensorMap tq, tk, tv;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, 64)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 64)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, kv_box_rows)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, kv_box_rows)) != SPARSED_OK) return st;
   AttnParams p;
   p.o = o;
   p.o_stride_b = rs.o[0];
@@ -316,6 +360,8 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   p.o_stride_t = rs.o[2];
   p.lse = lse_or_null;
   p.tile_lse = tile_lse_or_null;
+  p.stat_keys = 64;
+  p.slow_path_events = reinterpret_cast<unsigned long long*>(static_cast<uint8_t*>(ws) + 32);
   p.seq_len = shape->seq_len;
   p.heads_q = shape->heads_q;
   p.group = shape->heads_q / shape->heads_kv;
@@ -361,11 +407,12 @@ sparsed_status sparsed_select_from_stats(const sparsed_shape* shape, const spars
   sparsed_status st = kept_counts(params, nb, &pb, &k_pre, &k_gen);
   if (st != SPARSED_OK) return st;
   if (lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (!aligned16(lse) || !aligned16(tile_stats) || !aligned16(scores_out_or_null)) return SPARSED_ERR_ALIGNMENT;
   // the recorded statistics are per 64 keys: 32-key blocks need sparsed_select_pattern
   if (shape->seq_len > 131072 || params->block_size == 32) return SPARSED_ERR_UNSUPPORTED;
   if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
     return st;
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
   PoolParams pp;
   pp.tile_lse = tile_stats;
@@ -392,7 +439,7 @@ sparsed_status sparsed_select_pattern_pooled_qk(const sparsed_shape* shape, cons
   if (st != SPARSED_OK) return st;
   if (params == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (q == nullptr || k == nullptr) return SPARSED_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k)) return SPARSED_ERR_ALIGNMENT;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(scores_out_or_null)) return SPARSED_ERR_ALIGNMENT;
   if (params->block_size != 32 && params->block_size != 64 && params->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (shape->seq_len % params->block_size != 0) return SPARSED_ERR_ALIGNMENT;
   const int nb = shape->seq_len / params->block_size;
@@ -403,7 +450,7 @@ sparsed_status sparsed_select_pattern_pooled_qk(const sparsed_shape* shape, cons
     return st;
   size_t need = 0;
   if ((st = sparsed_workspace_bytes(SPARSED_OP_SELECT_POOLED_QK, shape, params, &need)) != SPARSED_OK) return st;
-  if (ws == nullptr || ws_bytes < need) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_ws(ws, ws_bytes, need)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
   PooledQkParams p;
   p.q = q;
@@ -440,11 +487,12 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   if (q == nullptr || k == nullptr || v == nullptr || o == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SPARSED_ERR_ALIGNMENT;
   if (pattern == nullptr || pattern->row_ptr == nullptr || pattern->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if (!aligned4(pattern->row_ptr) || !aligned4(pattern->col_idx)) return SPARSED_ERR_ALIGNMENT;
   if (pattern->block_size != 32 && pattern->block_size != 64 && pattern->block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (pattern->batch != shape->batch || pattern->heads_q != shape->heads_q || pattern->num_blocks < 1 ||
       static_cast<int64_t>(pattern->num_blocks) * pattern->block_size != shape->seq_len)
     return SPARSED_ERR_PATTERN;
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
   const int bs = pattern->block_size;
   CUtensorMap tq, tk, tv;
@@ -459,6 +507,8 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   p.o_stride_t = rs.o[2];
   p.lse = nullptr;
   p.tile_lse = nullptr;
+  p.stat_keys = 64;
+  p.slow_path_events = reinterpret_cast<unsigned long long*>(static_cast<uint8_t*>(ws) + 32);
   p.seq_len = shape->seq_len;
   p.heads_q = shape->heads_q;
   p.group = shape->heads_q / shape->heads_kv;
@@ -475,10 +525,13 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params* params, c
                                           int32_t heads_q, int32_t num_blocks, sparsed_pattern* out, void* ws,
                                           size_t ws_bytes, void* cuda_stream) {
   if (scores == nullptr || batch < 1 || heads_q < 1 || num_blocks < 1) return SPARSED_ERR_INVALID_ARG;
+  if (!aligned16(scores)) return SPARSED_ERR_ALIGNMENT;
   int pb = 0, k_pre = 0, k_gen = 0;
   sparsed_status st = kept_counts(params, num_blocks, &pb, &k_pre, &k_gen);
   if (st != SPARSED_OK) return st;
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
+  if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if ((st = check_arch()) != SPARSED_OK) return st;
   return run_topk(scores, batch, heads_q, num_blocks, params->block_size, pb, k_pre, k_gen, out,
                   static_cast<cudaStream_t>(cuda_stream));
 }
@@ -496,7 +549,8 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   int pb = 0, k_pre = 0, k_gen = 0;
   if ((st = kept_counts(params, nb, &pb, &k_pre, &k_gen)) != SPARSED_OK) return st;
   if (q == nullptr || k == nullptr) return SPARSED_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k)) return SPARSED_ERR_ALIGNMENT;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(lse_or_null) || !aligned16(scores_out_or_null))
+    return SPARSED_ERR_ALIGNMENT;
   if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
     return st;
   // With few enough blocks per row the pooled-scoring kernel ranks each block-row in its own
@@ -507,7 +561,7 @@ sparsed_status sparsed_select_pattern(const sparsed_shape* shape, const sparsed_
   const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
   const bool need_score_ws = !fused && scores_out_or_null == nullptr;
   const size_t required = SPARSED_STATUS_BYTES + (need_score_ws ? score_bytes : 0) + (lse_or_null ? 0 : lse_bytes);
-  if (ws == nullptr || ws_bytes < required) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_ws(ws, ws_bytes, required)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* base = static_cast<uint8_t*>(ws);
@@ -560,7 +614,7 @@ sparsed_status sparsed_attention_step(const sparsed_shape* shape, const sparsed_
   size_t need = 0;
   sparsed_status st = sparsed_workspace_bytes(SPARSED_OP_ATTENTION_STEP, shape, params, &need);
   if (st != SPARSED_OK) return st;
-  if (ws == nullptr || ws_bytes < need) return SPARSED_ERR_WORKSPACE;
+  if ((st = check_ws(ws, ws_bytes, need)) != SPARSED_OK) return st;
   const size_t bh = static_cast<size_t>(shape->batch) * shape->heads_q;
   const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
   uint8_t* base = static_cast<uint8_t*>(ws);
@@ -579,6 +633,29 @@ sparsed_status sparsed_attention_step(const sparsed_shape* shape, const sparsed_
                                 cuda_stream);
 }
 
+sparsed_status sparsed_attention_step_variant(const sparsed_shape* shape, const sparsed_select_params* params,
+                                              int32_t variant, int32_t step_1based, int32_t total_steps, double skip,
+                                              const void* q, const void* k, const void* v, void* o,
+                                              sparsed_pattern* pattern, void* ws, size_t ws_bytes, void* cuda_stream,
+                                              int32_t* mode_out_or_null) {
+  if (params == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if ((variant & ~(SPARSED_VARIANT_NO_REUSE | SPARSED_VARIANT_NO_ISOLATION)) != 0) return SPARSED_ERR_INVALID_ARG;
+  sparsed_select_params p2 = *params;
+  if (variant & SPARSED_VARIANT_NO_ISOLATION) p2.prefill_len = 0;
+  const int32_t mode = sparsed_schedule_mode(step_1based, total_steps, skip);
+  if (mode < 0) return SPARSED_ERR_INVALID_ARG;
+  if (mode == SPARSED_MODE_SPARSE && (variant & SPARSED_VARIANT_NO_REUSE)) {
+    // "without Sparse Reusing": this step's own Q and K give this step's pattern (row statistics
+    // pass + pooled scoring + ranking), then the block-sparse attention runs on it
+    if (mode_out_or_null != nullptr) *mode_out_or_null = mode;
+    sparsed_status st = sparsed_select_pattern(shape, &p2, q, k, nullptr, pattern, nullptr, ws, ws_bytes, cuda_stream);
+    if (st != SPARSED_OK) return st;
+    return sparsed_attn_sparse(shape, pattern, q, k, v, o, ws, ws_bytes, cuda_stream);
+  }
+  return sparsed_attention_step(shape, &p2, step_1based, total_steps, skip, q, k, v, o, pattern, ws, ws_bytes,
+                                cuda_stream, mode_out_or_null);
+}
+
 sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int32_t num_blocks, int32_t block_size,
                                             int32_t sink_blocks, int32_t window_blocks, sparsed_pattern* out,
                                             void* cuda_stream) {
@@ -586,6 +663,7 @@ sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int3
   if (block_size != 32 && block_size != 64 && block_size != 128) return SPARSED_ERR_UNSUPPORTED;
   if (num_blocks > 16384) return SPARSED_ERR_UNSUPPORTED;
   if (out == nullptr || out->row_ptr == nullptr || out->col_idx == nullptr) return SPARSED_ERR_PATTERN;
+  if (!aligned4(out->row_ptr) || !aligned4(out->col_idx)) return SPARSED_ERR_ALIGNMENT;
   const int sink = sink_blocks < num_blocks ? sink_blocks : num_blocks;
   const int half = (window_blocks - 1) / 2;
   const int64_t per_head = window_pattern_nnz_per_head(num_blocks, sink, half);
@@ -607,7 +685,9 @@ sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int3
 sparsed_status sparsed_pattern_validate(const sparsed_pattern* pattern, void* ws, size_t ws_bytes, void* cuda_stream) {
   if (pattern == nullptr || pattern->row_ptr == nullptr || pattern->col_idx == nullptr) return SPARSED_ERR_PATTERN;
   if (pattern->batch < 1 || pattern->heads_q < 1 || pattern->num_blocks < 1) return SPARSED_ERR_PATTERN;
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
+  if (!aligned4(pattern->row_ptr) || !aligned4(pattern->col_idx)) return SPARSED_ERR_ALIGNMENT;
+  sparsed_status st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES);
+  if (st != SPARSED_OK) return st;
   const int64_t rows = static_cast<int64_t>(pattern->batch) * pattern->heads_q * pattern->num_blocks;
   if (rows >= INT32_MAX) return SPARSED_ERR_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -626,15 +706,16 @@ sparsed_status sparsed_pattern_validate(const sparsed_pattern* pattern, void* ws
 }
 
 sparsed_status sparsed_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream) {
-  if (ws == nullptr || ws_bytes < SPARSED_STATUS_BYTES) return SPARSED_ERR_WORKSPACE;
-  sparsed_status st = check_arch();
+  sparsed_status st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES);
   if (st != SPARSED_OK) return st;
+  if ((st = check_arch()) != SPARSED_OK) return st;
   cudaError_t e = launch_wait_timeout_selftest(static_cast<DeviceStatus*>(ws), 99, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
 sparsed_status sparsed_last_device_status(void* ws, void* cuda_stream, int32_t* code, int32_t* where) {
   if (ws == nullptr) return SPARSED_ERR_WORKSPACE;
+  if (!aligned4(ws)) return SPARSED_ERR_ALIGNMENT;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   int32_t host[2] = {0, 0};
   cudaError_t e = cudaMemcpyAsync(host, ws, sizeof(host), cudaMemcpyDeviceToHost, stream);

@@ -10,7 +10,11 @@
 //                             O += P_j V_j with P read from tensor memory (P overwrites the
 //                             first half of S_j's columns). S_{j+1} is issued before P_j V_j,
 //                             so the tensor pipe works on the next logits while the softmax
-//                             warps are busy with the current ones.
+//                             warps are busy with the current ones. Each batch of MMAs ends in ONE
+//                             commit to the barrier of the ring slot it read: that barrier tells the
+//                             softmax warps "S_j is ready" / "P_j V_j has drained" and the producer
+//                             "the slot is free" (the issuing thread is the pipeline's bottleneck:
+//                             a commit costs it about 150 clocks, a barrier poll about 100).
 //   warps 0-3: one thread per query row - online softmax in fp32 on base-2 logits. The tile
 //             is exponentiated once against the running maximum; only if a row sum shows that
 //             logits may have outgrown it by more than 2^8 is the tile redone with the new
@@ -20,6 +24,7 @@
 // consecutive tiles, two 32-key blocks share one). Two CTAs fit on one SM (112 KB of shared memory
 // and 256 tensor-memory columns each).
 #include "internal.h"
+#include "softmax_pipeline.cuh"
 
 namespace sparsed {
 namespace {
@@ -51,8 +56,9 @@ constexpr int kPolyEvery = SPARSED_ATTN_POLY_EVERY;  // every n-th exponential o
 struct AttnSmem {
   alignas(1024) __nv_bfloat16 q[2][kTileM * 64];           // two 64-wide halves of head_dim
   alignas(1024) __nv_bfloat16 kv[kSlots][2][kTileN * 64];  // each slot: two 64-wide halves of head_dim
-  uint64_t q_full, kv_full[kSlots], kv_empty[kSlots];
-  uint64_t s_full[2], p_full[2], o_full;
+  uint64_t q_full, kv_full[kSlots];
+  uint64_t done[kSlots];   // the MMAs that read the slot have completed (Q K^T for a K tile, P V for a V tile)
+  uint64_t p_full[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -116,13 +122,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(&sm.kv_full[s], 1);
-      mbar_init(&sm.kv_empty[s], 1);
+      mbar_init(&sm.done[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.s_full[s], 1);
-      mbar_init(&sm.p_full[s], kSoftmaxThreads);
-    }
-    mbar_init(&sm.o_full, 1);
+    for (int s = 0; s < 2; ++s) mbar_init(&sm.p_full[s], kSoftmaxThreads);
     sm.abort_flag = 0;
     mbar_fence_init();
   }
@@ -187,7 +189,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const int slot = i % kSlots;
           TL(20 + which);
           if (i >= kSlots) {
-            ok = mbar_wait(&sm.kv_empty[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
+            ok = mbar_wait(&sm.done[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
           }
@@ -216,16 +218,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   } else if (warp == 5) {
     // =============================== UMMA issuer ========================================
     if (num_tiles > 0) {
-      constexpr uint32_t idesc_qk = umma_idesc_bf16(kTileM, kTileN, false, false);
-      constexpr uint32_t idesc_pv = umma_idesc_bf16(kTileM, kHeadDim, false, true);
-      constexpr uint32_t hi_desc = umma_desc_hi_sw128(1024);
       // descriptor low words: Q is fixed; K/V slots differ only in their base address
       const uint32_t q_lo0 = umma_desc_lo(smem_u32(sm.q[0]), 16);
       const uint32_t kv_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), 16);            // as K (K-major)
       const uint32_t v_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), kTileN * 128);   // as V (MN-major)
-      constexpr uint32_t q_half_step = (kTileM * 64 * 2) >> 4;                    // 16 KB per head_dim half of Q
       constexpr uint32_t slot_step = (2 * kTileN * 64 * 2) >> 4;                  // 16 KB per ring slot
-      constexpr uint32_t half_step = (kTileN * 64 * 2) >> 4;                      // 8 KB per head_dim half
       TL_DECL(1)
       // S_t = Q K_t^T into S buffer t & 1
       auto issue_qk = [&](int t) -> bool {
@@ -236,20 +233,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         got = __all_sync(0xffffffffu, got);
         if (!got) return false;
         TL(11);
-        tc_fence_after();
-        if (elect_one_sync()) {
-          const uint32_t k_lo = kv_lo0 + slot * slot_step;
-          const uint32_t tS = tmem + kColS + (t & 1) * kTileN;
-          umma_ss_words<false>(tS, q_lo0, hi_desc, k_lo, hi_desc, idesc_qk);
-#pragma unroll
-          for (int kk = 1; kk < kHeadDim / 16; ++kk) {
-            umma_ss_words<true>(tS, q_lo0 + (kk >> 2) * q_half_step + (kk & 3) * 2, hi_desc,
-                                k_lo + (kk >> 2) * half_step + (kk & 3) * 2, hi_desc, idesc_qk);
-          }
-          umma_commit(&sm.kv_empty[slot]);
-          umma_commit(&sm.s_full[t & 1]);
-        }
-        __syncwarp();
+        issue_qk64(tmem + kColS + (t & 1) * kTileN, q_lo0, kv_lo0 + slot * slot_step, &sm.done[slot]);
         TL(12);
         return true;
       };
@@ -262,25 +246,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (t + 1 < num_tiles && !issue_qk(t + 1)) break;
         const int i = 2 * t + 1;
         const int slot = i % kSlots;
-        ok = mbar_wait(&sm.p_full[t & 1], (t >> 1) & 1, &sm.abort_flag, p.status, 22);
         TL(13);
-        ok = ok && mbar_wait(&sm.kv_full[slot], (i / kSlots) & 1, &sm.abort_flag, p.status, 23);
+        ok = mbar_wait2(&sm.p_full[t & 1], (t >> 1) & 1, &sm.kv_full[slot], (i / kSlots) & 1, &sm.abort_flag,
+                        p.status, 22);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         TL(14);
-        tc_fence_after();
-        if (elect_one_sync()) {
-          const uint32_t v_lo = v_lo0 + slot * slot_step;
-          const uint32_t tP = tmem + kColS + (t & 1) * kTileN;
-          // V tile is [key][d]: MN-major B operand; 16 keys per step are 2048 bytes apart
-          umma_ts_words(tO, tP, v_lo, hi_desc, idesc_pv, t > 0 ? 1u : 0u);
-#pragma unroll
-          for (int kk = 1; kk < kTileN / 16; ++kk)
-            umma_ts_words(tO, tP + kk * 8, v_lo + kk * 128, hi_desc, idesc_pv, 1u);
-          umma_commit(&sm.kv_empty[slot]);
-          if (t == num_tiles - 1) umma_commit(&sm.o_full);
-        }
-        __syncwarp();
+        issue_pv64(tO, tmem + kColS + (t & 1) * kTileN, v_lo0 + slot * slot_step, t > 0, &sm.done[slot]);
         TL(15);
       }
     }
@@ -288,8 +260,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     // =============================== softmax / epilogue =================================
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     const float scale_log2 = p.scale_log2;
-    float m_used = -INFINITY;
-    float l = 0.f;
     bool ok = true;
     TL_DECL(0)
 #ifdef SPARSED_TIMELINE
@@ -297,9 +267,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #undef TL
 #define TL(tag) do { if (tl_on2 && tl_n < 2047) { tl_buf[1 + tl_n++] = (static_cast<long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFll); tl_buf[0] = tl_n; } } while (0)
 #endif
+    RowState st{-INFINITY, 0.f};
     for (int t = 0; t < num_tiles; ++t) {
       TL(1);
-      if (!mbar_wait(&sm.s_full[t & 1], (t >> 1) & 1, &sm.abort_flag, p.status, 30)) {
+      // S_t is ready when the Q K^T batch that read ring slot 2t has completed
+      if (!mbar_wait(&sm.done[(2 * t) % kSlots], ((2 * t) / kSlots) & 1, &sm.abort_flag, p.status, 30)) {
         ok = false;
         break;
       }
@@ -314,87 +286,27 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if constexpr (kBlocksPerTile > 1) {
         // only the last tile can be ragged: an odd block list leaves its second half empty
         const int valid_cols = (list_len - kBlocksPerTile * t) * kBlock;
-        if (valid_cols < kTileN) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (j >= valid_cols) r0[j] = 0xff800000u;       // -inf
-            if (32 + j >= valid_cols) r1[j] = 0xff800000u;
-          }
-        }
+        if (valid_cols < kTileN) mask_columns_from(r0, r1, valid_cols);
       }
-      // Fast path: one pass against the running maximum m, p = 2^(s*scale - m), with packed
-      // fp32x2 arithmetic. No row maximum is taken here: if every p were above 2^8 the row sum
-      // would exceed 2^8 too, so a sum <= 2^8 proves that the stale maximum is still safe.
       uint32_t pk[32];
-      float sum;
-      {
-        const float2 sc = make_float2(scale_log2, scale_log2);
-        const float2 nm = make_float2(-m_used, -m_used);
-        float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(r0[2 * j]), __uint_as_float(r0[2 * j + 1])), sc, nm);
-          const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(r1[2 * j]), __uint_as_float(r1[2 * j + 1])), sc, nm);
-          const float2 e0 = make_float2(tile_exp2<kPolyEvery>(x0.x, 2 * j), tile_exp2<kPolyEvery>(x0.y, 2 * j + 1));
-          const float2 e1 = make_float2(tile_exp2<kPolyEvery>(x1.x, 2 * j), tile_exp2<kPolyEvery>(x1.y, 2 * j + 1));
-          acc0 = __fadd2_rn(acc0, e0);
-          acc1 = __fadd2_rn(acc1, e1);
-          pk[j] = pack_bf16x2(e0.x, e0.y);
-          pk[16 + j] = pack_bf16x2(e1.x, e1.y);
-        }
-        sum = (acc0.x + acc0.y) + (acc1.x + acc1.y);
-      }
-      const bool trigger = !(sum <= 256.0f);  // also true on the first tile (m = -inf) and for NaN
+      float2 sums = softmax_group_fast<kPolyEvery>(r0, r1, scale_log2, st.m, pk);
+      const bool trigger = !(sums.x + sums.y <= 256.0f);  // also true on the first tile (m = -inf) and for NaN
       if (__any_sync(0xffffffffu, trigger)) {
-        // Slow path (first tile, or logits that outgrew the running maximum): take the true row
-        // maximum, adopt it where it grew, redo the tile and rescale what O holds so far.
-        float mx = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, fmaxf(__uint_as_float(r0[j]), __uint_as_float(r1[j])));
-        const float m_tile = mx * scale_log2;
-        float alpha = 1.f;
-        if (m_tile > m_used) {
-          alpha = fast_exp2(m_used - m_tile);  // 0 on the first tile
-          m_used = m_tile;
-          l *= alpha;
-        }
-        sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(r0[2 * j]), scale_log2, -m_used));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(r0[2 * j + 1]), scale_log2, -m_used));
-          sum += p0;
-          sum += p1;
-          pk[j] = pack_bf16x2(p0, p1);
-        }
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(r1[2 * j]), scale_log2, -m_used));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(r1[2 * j + 1]), scale_log2, -m_used));
-          sum += p0;
-          sum += p1;
-          pk[16 + j] = pack_bf16x2(p0, p1);
-        }
+        // first tile, or logits that outgrew the running maximum
+        const float alpha = softmax_group_exact(r0, r1, scale_log2, st, pk, sums);
         if (t > 0) {
-          // O must be quiescent: wait until P_{t-1} V_{t-1} has drained (its ring slot was released)
-          const int ip = 2 * (t - 1) + 1;  // the load index of V_{t-1}
-          if (!mbar_wait(&sm.kv_empty[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
+          // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring slot 2t-1) has drained
+          const int ip = 2 * (t - 1) + 1;
+          if (!mbar_wait(&sm.done[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
             ok = false;
             break;
           }
           tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < kHeadDim / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tO + lane_base + c * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-            tmem_st32(tO + lane_base + c * 32, o);
-          }
+          rescale_accumulator_row(tO + lane_base, alpha);
+          if (p.slow_path_events != nullptr && (tid & 31) == 0) atomicAdd(p.slow_path_events, 1ull);
         }
       }
-      l += sum;
+      st.l += sums.x + sums.y;
       TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();
@@ -404,37 +316,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
 
     // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
-    if (ok && num_tiles > 0) ok = mbar_wait(&sm.o_full, 0, &sm.abort_flag, p.status, 31);
+    if (ok && num_tiles > 0) {
+      const int il = 2 * (num_tiles - 1) + 1;   // the last P V read ring slot il
+      ok = mbar_wait(&sm.done[il % kSlots], (il / kSlots) & 1, &sm.abort_flag, p.status, 31);
+    }
     tc_fence_after();
     const int row_in_tile = tid;
     const int row = q_row0 + row_in_tile;
     const bool row_valid = (row_in_tile < kRowsQ) && (row < p.seq_len);
-    const float inv_l = (num_tiles > 0) ? (1.f / l) : 0.f;
+    const float inv_l = (num_tiles > 0) ? (1.f / st.l) : 0.f;
     __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + batch * p.o_stride_b + head * p.o_stride_h +
                            static_cast<int64_t>(row) * p.o_stride_t;
-#pragma unroll
-    for (int c = 0; c < kHeadDim / 32; ++c) {
-      uint32_t r[32];
-      if (num_tiles > 0) {
-        tmem_ld32(tO + lane_base + c * 32, r);
-        tmem_wait_ld();
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) r[j] = 0u;
-      }
-      if (row_valid) {
-        uint4* dst = reinterpret_cast<uint4*>(o_row + c * 32);
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint4 out;
-          out.x = pack_bf16x2(__uint_as_float(r[8 * g + 0]) * inv_l, __uint_as_float(r[8 * g + 1]) * inv_l);
-          out.y = pack_bf16x2(__uint_as_float(r[8 * g + 2]) * inv_l, __uint_as_float(r[8 * g + 3]) * inv_l);
-          out.z = pack_bf16x2(__uint_as_float(r[8 * g + 4]) * inv_l, __uint_as_float(r[8 * g + 5]) * inv_l);
-          out.w = pack_bf16x2(__uint_as_float(r[8 * g + 6]) * inv_l, __uint_as_float(r[8 * g + 7]) * inv_l);
-          dst[g] = out;
-        }
-      }
-    }
+    store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
   }
 
   // ---- teardown ------------------------------------------------------------------------
@@ -451,14 +344,9 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
                    int batch, cudaStream_t stream) {
   auto kernel = attn_kernel<kBlock, kRowsQ>;
   const int smem = static_cast<int>(sizeof(AttnSmem));
-  static bool configured[64] = {};  // per template instantiation and device
-  int dev = 0;
-  cudaGetDevice(&dev);
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) configured[dev] = true;
-  }
+  static SmemLimit limit;  // per template instantiation
+  cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
+  if (e != cudaSuccess) return e;
   const long long ctas = static_cast<long long>(batch) * p.heads_q * p.num_q_tiles;
   if (ctas <= 0) return cudaSuccess;
   kernel<<<static_cast<unsigned>(ctas), kThreads, smem, stream>>>(tq, tk, tv, p);

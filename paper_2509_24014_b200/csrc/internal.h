@@ -5,16 +5,43 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "sm100_primitives.cuh"
 
 namespace sparsed {
+
+// Per-kernel record of the dynamic shared-memory limit already granted on each device, so that
+// cudaFuncSetAttribute runs once per (kernel, device) instead of on every launch. Safe to use from
+// several host threads: the fast path is one atomic load, the slow path is serialised.
+struct SmemLimit {
+  std::atomic<int> granted[64];
+  std::mutex slow;
+};
+
+template <class Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, SmemLimit& lim) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && lim.granted[dev].load(std::memory_order_acquire) >= bytes) return cudaSuccess;
+  std::lock_guard<std::mutex> lock(lim.slow);
+  if (tracked && lim.granted[dev].load(std::memory_order_relaxed) >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && tracked) lim.granted[dev].store(bytes, std::memory_order_release);
+  return e;
+}
 
 // Parameters shared by the dense and the block-sparse attention kernels.
 struct AttnParams {
   void* o;                 // bf16 [B,Hq,L,D]
   int64_t o_stride_b, o_stride_h, o_stride_t;
   float* lse;              // fp32 [B,Hq,L] or null
-  float* tile_lse;         // fp32 [B*Hq, ceil(L/128), ceil(L/64), 128] or null: base-2 log-sum-exp of each row over each 64-key tile
+  float* tile_lse;         // fp32 [B*Hq, ceil(L/128), ceil(L/stat_keys), 128] or null: base-2 log-sum-exp of each row over each group of stat_keys keys
+  int stat_keys;           // 32, 64 or 128
+  unsigned long long* slow_path_events;  // counts warp-level rescales of the output accumulator, or null
   int seq_len;
   int heads_q;
   int group;               // heads_q / heads_kv
@@ -32,7 +59,7 @@ struct ScoreParams {
   int seq_len;
   int heads_q;
   int group;
-  int block_size;          // 64 or 128
+  int block_size;          // 32, 64 or 128
   float scale_log2;
   DeviceStatus* status;
   // fused selection (row_ptr != null): each CTA ranks the block-row(s) it has just pooled

@@ -175,7 +175,8 @@ cudaError_t launch_pool_select(const PoolParams& p, cudaStream_t stream) {
   const int n_tiles = (p.seq_len + 63) / 64;
   if (n_tiles > kMaxTiles) return cudaErrorInvalidValue;
   const int smem = static_cast<int>(pool_smem_bytes(n_tiles, p.seq_len / p.block_size));
-  cudaError_t e = cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  static SmemLimit limit;
+  cudaError_t e = ensure_dynamic_smem(pool_select_kernel, smem, limit);
   if (e != cudaSuccess) return e;
   const int num_q_tiles = (p.seq_len + kRows - 1) / kRows;
   const long long ctas = static_cast<long long>(p.bh) * num_q_tiles;

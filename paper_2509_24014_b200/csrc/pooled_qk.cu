@@ -212,8 +212,8 @@ cudaError_t launch_pooled_qk_select(const PooledQkParams& p, cudaStream_t stream
   if (e != cudaSuccess) return e;
   const size_t smem = SelectSmemLayout::bytes(p.nb);
   if (smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(pooled_qk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
+    static SmemLimit limit;
+    e = ensure_dynamic_smem(pooled_qk_select_kernel, static_cast<int>(smem), limit);
     if (e != cudaSuccess) return e;
   }
   const int row_tiles = (p.nb + kRowsPerCta - 1) / kRowsPerCta;

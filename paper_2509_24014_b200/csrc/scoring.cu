@@ -290,7 +290,8 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScorePara
                    cudaStream_t stream) {
   auto kernel = score_kernel<kStatsOnly>;
   const int smem = static_cast<int>(sizeof(ScoreSmem));
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  static SmemLimit limit;  // per template instantiation
+  cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
   if (e != cudaSuccess) return e;
   const int num_q_tiles = (p.seq_len + kTile - 1) / kTile;
   const long long ctas = static_cast<long long>(batch) * p.heads_q * num_q_tiles;

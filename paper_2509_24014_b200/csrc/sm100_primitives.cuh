@@ -89,6 +89,28 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+// Bounded wait on two barriers at once: both polls are issued before either result is looked at,
+// so their latencies overlap (a poll of a barrier in shared memory costs on the order of 100 clocks
+// even when it succeeds).
+__device__ __forceinline__ bool mbar_wait2(uint64_t* bar_a, uint32_t parity_a, uint64_t* bar_b, uint32_t parity_b,
+                                           volatile int* abort_flag, DeviceStatus* status, int where,
+                                           uint32_t limit = kSpinLimit) {
+  bool a = false, b = false;
+  for (uint32_t it = 0; it < limit; ++it) {
+    const bool ta = a || mbar_try_wait(bar_a, parity_a);
+    const bool tb = b || mbar_try_wait(bar_b, parity_b);
+    a = ta;
+    b = tb;
+    if (a && b) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  if (status != nullptr) {
+    if (atomicCAS(&status->code, 0, 1) == 0) status->where = where;
+  }
+  return false;
+}
+
 // ----------------------------------------------------------------------------
 // Proxy fences
 // ----------------------------------------------------------------------------

@@ -91,8 +91,8 @@ cudaError_t launch_topk_csr(const TopkParams& p, cudaStream_t stream) {
   const int nb_pad = (p.nb + 3) & ~3;
   const size_t smem = static_cast<size_t>(warps) * (nb_pad + 256) * 4;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(topk_csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
+    static SmemLimit limit;
+    cudaError_t e = ensure_dynamic_smem(topk_csr_kernel, static_cast<int>(smem), limit);
     if (e != cudaSuccess) return e;
   }
   const unsigned ctas = static_cast<unsigned>((p.rows + warps - 1) / warps);

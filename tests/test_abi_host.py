@@ -93,6 +93,37 @@ def test_argument_errors_are_status_codes(lib):
     assert binding.status_string(5) == "pattern invalid or too small"
 
 
+def test_misaligned_side_buffers_are_refused_before_any_launch(lib):
+    """fp32 side buffers (LSE, tile statistics, scores, workspace) are read with 16-byte loads and the
+    CSR arrays as int32: a pointer offset by 4 (or 2) bytes must come back as an alignment error from
+    the host-side checks, with nothing launched (there is no GPU here to launch on)."""
+    shape = binding.Shape(1, 2, 2, 1024, 128)
+    params = sd.make_params(128, 0.25, 0)
+    ok, off = 4096, 4096 + 4
+    pat = binding.Pattern(ok, ok, 1 << 20, 0, 0, 0, 0, 0)
+    byref = ctypes.byref
+    assert lib.sparsed_attn_full(byref(shape), ok, ok, ok, ok, off, ok, 256, None) == 3             # lse
+    assert lib.sparsed_attn_full(byref(shape), ok, ok, ok, ok, None, off, 256, None) == 3            # ws
+    assert lib.sparsed_attn_full_stats(byref(shape), ok, ok, ok, ok, ok, off, ok, 256, None) == 3    # tile stats
+    assert lib.sparsed_select_from_stats(byref(shape), byref(params), off, ok, byref(pat), None, ok, 256, None) == 3
+    assert lib.sparsed_select_from_stats(byref(shape), byref(params), ok, off, byref(pat), None, ok, 256, None) == 3
+    assert lib.sparsed_select_from_stats(byref(shape), byref(params), ok, ok, byref(pat), off, ok, 256, None) == 3
+    assert lib.sparsed_select_from_stats(byref(shape), byref(params), ok, ok, byref(pat), None, off, 256, None) == 3
+    assert lib.sparsed_select_from_scores(byref(params), off, 1, 2, 8, byref(pat), ok, 256, None) == 3
+    assert lib.sparsed_select_from_scores(byref(params), ok, 1, 2, 8, byref(pat), off, 256, None) == 3
+    big = 1 << 24
+    assert lib.sparsed_select_pattern(byref(shape), byref(params), ok, ok, off, byref(pat), None, ok, big, None) == 3
+    assert lib.sparsed_select_pattern(byref(shape), byref(params), ok, ok, None, byref(pat), off, ok, big, None) == 3
+    assert lib.sparsed_select_pattern(byref(shape), byref(params), ok, ok, None, byref(pat), None, off, big, None) == 3
+    assert lib.sparsed_select_pattern_pooled_qk(byref(shape), byref(params), ok, ok, byref(pat), off, ok, big, None) == 3
+    assert lib.sparsed_select_pattern_pooled_qk(byref(shape), byref(params), ok, ok, byref(pat), None, off, big, None) == 3
+    bad_pat = binding.Pattern(ok + 2, ok, 1 << 20, 0, 128, 8, 1, 2)
+    assert lib.sparsed_attn_sparse(byref(shape), byref(bad_pat), ok, ok, ok, ok, ok, 256, None) == 3
+    assert lib.sparsed_select_from_stats(byref(shape), byref(params), ok, ok, byref(bad_pat), None, ok, 256, None) == 3
+    assert lib.sparsed_workspace_init(off, 256, None) == 3
+    assert lib.sparsed_pattern_validate(byref(binding.Pattern(ok, ok + 2, 16, 16, 128, 8, 1, 2)), ok, 256, None) == 3
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding._build, "LIB_PATH", str(tmp_path / "nope.so"))

@@ -62,6 +62,47 @@ def test_schedule_through_one_entry_point(bs, L, rho, prefill, T, skip):
     assert sd.sparsed_last_device_status(ws) == (0, 0)
 
 
+def test_schedule_at_config2_size_sampled():
+    """The LLaDA-shaped 8k layer (32 heads, 4096 prompt + 4096 generation tokens) through the one-call
+    entry point, with fresh noise each step: step 1 full, step 2 full + selection from that pass's row
+    statistics, steps 3-4 sparse on the kept pattern. The oracle follows on sampled (head, query block)
+    rows, including the two blocks next to the prompt boundary."""
+    from tests.test_gpu_parity_configs import check_row_list
+    cfg = syn.CONFIGS["c2"].with_(total_steps=4, skip=0.5, step_noise=0.05)
+    T, skip, bs, nb, pb = 4, 0.5, cfg.block_size, cfg.num_blocks, cfg.prefill_len // cfg.block_size
+    base = syn.make_base(cfg, DEV)
+    params = sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)
+    kp, kg = sd.sparsed_kept_per_row(params, cfg.seq_len)
+    assert (kp, kg) == (7, 7)
+    pat, rp_t, ci_t = sd.new_pattern(1, cfg.heads_q, nb, kp + kg, DEV)
+    q0, k0, _ = syn.make_qkv(cfg, DEV, step=1, base=base)
+    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_ATTENTION_STEP, sd.make_shape(q0, k0), params), DEV)
+    heads, blocks = (0, 13, 31), (0, pb - 1, pb, nb - 1)
+    rp = ci = None
+    for step in range(1, T + 1):
+        q, k, v = syn.make_qkv(cfg, DEV, step=step, base=base)
+        o = torch.empty_like(q)
+        mode = sd.sparsed_attention_step(q, k, v, o, params, step, T, skip, pat, ws)
+        torch.cuda.synchronize()
+        assert mode == orc.schedule_mode(step, T, skip)
+        if step == 2:
+            rp, ci = rp_t.cpu().numpy(), ci_t.cpu().numpy()
+            assert pat.nnz == 32 * nb * 14 and sd.sparsed_pattern_validate(pat, sd.new_workspace(256, DEV))
+        for h in heads:
+            qh, kh, vh = to_f64(q[0, h]), to_f64(k[0, h]), to_f64(v[0, h])
+            for ib in blocks:
+                rows = slice(ib * bs, (ib + 1) * bs)
+                r = h * nb + ib
+                if mode != sd.MODE_SPARSE:
+                    check_outputs(o[0, h, rows], orc.head_full_rows(qh, kh, vh, rows)[0], f"step {step} full h{h} ib{ib}")
+                    if mode == sd.MODE_FULL_AND_SELECT:
+                        check_row_list(ci[rp[r]:rp[r + 1]], orc.head_pooled_row(qh, kh, ib, bs), pb, cfg.keep_ratio)
+                else:
+                    ref = orc.head_sparse_rows(qh, kh, vh, ib, ci[rp[r]:rp[r + 1]], bs)
+                    check_outputs(o[0, h, rows], ref, f"step {step} sparse h{h} ib{ib}")
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+
+
 def test_step_argument_checks():
     cfg = syn.AttnConfig("step", 1, 1, 1, 256, 128, 128, 0.5, 0, seed=1)
     q, k, v = syn.make_qkv(cfg, DEV)

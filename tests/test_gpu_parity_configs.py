@@ -58,12 +58,37 @@ def sample_blocks(nb, pb, n, rng):
     return sorted(fixed | set(rest[: max(0, n - len(fixed))]))
 
 
-def check_sampled(cfg, q, k, v, heads, n_blocks, seed, what):
-    """Full, select and sparse on the GPU at full size; the oracle on sampled row blocks."""
+def gpu_switch_step_from_stats(q, k, v, block_size, keep_ratio, prefill_len):
+    """The switch step the way the benchmark and sparsed_attention_step run it: full attention that
+    records per-tile row statistics, then pooling + ranking from those statistics."""
+    B, Hq, L, _ = q.shape
+    nb = L // block_size
+    o = torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=q.device)
+    stats = sd.new_tile_stats(q)
+    ws = sd.new_workspace(256, q.device)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+    params = sd.make_params(block_size, keep_ratio, prefill_len)
+    kp, kg = sd.sparsed_kept_per_row(params, L)
+    pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, kp + kg, q.device)
+    scores = torch.full((B, Hq, nb, nb), float("nan"), dtype=torch.float32, device=q.device)
+    sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws, scores_out=scores)
+    torch.cuda.synchronize()
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+    return o, lse, pat, row_ptr, col_idx, scores
+
+
+def check_sampled(cfg, q, k, v, heads, n_blocks, seed, what, via_stats=False):
+    """Full, select and sparse on the GPU at full size; the oracle on sampled row blocks.
+    via_stats: select from the full pass's row statistics (the benchmarked path) instead of the
+    two-pass scorer."""
     bs, nb, pb = cfg.block_size, cfg.num_blocks, cfg.prefill_len // cfg.block_size
     group = cfg.heads_q // cfg.heads_kv
-    o, lse = gpu_full(q, k, v)
-    pat, row_ptr, col_idx, scores = gpu_select(q, k, bs, cfg.keep_ratio, cfg.prefill_len, lse=lse)
+    if via_stats:
+        o, lse, pat, row_ptr, col_idx, scores = gpu_switch_step_from_stats(q, k, v, bs, cfg.keep_ratio, cfg.prefill_len)
+    else:
+        o, lse = gpu_full(q, k, v)
+        pat, row_ptr, col_idx, scores = gpu_select(q, k, bs, cfg.keep_ratio, cfg.prefill_len, lse=lse)
     o_sp = gpu_sparse(q, k, v, pat)
     rp, ci = row_ptr.cpu().numpy(), col_idx.cpu().numpy()
     rng = np.random.default_rng(seed)
@@ -127,22 +152,27 @@ def test_config2_exhaustive():
     print({kk: float(np.mean(vv)) for kk, vv in by_kind.items()}, "rows that had to match exactly")
 
 
-def test_config3_gqa_sampled():
+@pytest.mark.parametrize("via_stats", [False, True], ids=["two_pass", "from_stats"])
+def test_config3_gqa_sampled(via_stats):
     cfg = syn.CONFIGS["c3"]
     q, k, v = syn.make_qkv(cfg, DEV)
-    n_exact, n_rows, worst, _ = check_sampled(cfg, q, k, v, range(cfg.heads_q), 4, 3, "c3")
+    n_exact, n_rows, worst, _ = check_sampled(cfg, q, k, v, range(cfg.heads_q), 4, 3, "c3", via_stats=via_stats)
     assert n_rows == 28 * 4 and worst <= 2e-2
 
 
-def test_config4_pattern_reuse_at_64k():
-    """Pattern selected at the switch step's tensors, reused on a later step's noisy tensors."""
+@pytest.mark.parametrize("via_stats", [False, True], ids=["two_pass", "from_stats"])
+def test_config4_pattern_reuse_at_64k(via_stats):
+    """Pattern selected at the switch step's tensors, reused on a later step's noisy tensors; once
+    through the two-pass scorer and once through the row statistics of the full pass (1024 key tiles
+    per row: the path the benchmark times)."""
     cfg = syn.CONFIGS["c4"]
     s = sd.sparsed_switch_step(cfg.total_steps, cfg.skip)
     assert s == 12 and sd.sparsed_schedule_mode(s, cfg.total_steps, cfg.skip) == sd.MODE_FULL_AND_SELECT
     base = syn.make_base(cfg, DEV)
     q, k, v = syn.make_qkv(cfg, DEV, step=s, base=base)
     heads = [0, 5, 13, 31]
-    n_exact, n_rows, worst, (_, _, pat, row_ptr, col_idx) = check_sampled(cfg, q, k, v, heads, 3, 4, "c4 step 12")
+    n_exact, n_rows, worst, (_, _, pat, row_ptr, col_idx) = check_sampled(cfg, q, k, v, heads, 3, 4, "c4 step 12",
+                                                                          via_stats=via_stats)
     assert pat.nnz == 32 * 512 * 52
     del q, k, v
     # final step: new noise, same pattern (Sparse Reusing)
@@ -160,8 +190,10 @@ def test_config4_pattern_reuse_at_64k():
             check_outputs(o_sp[0, h, ib * bs:(ib + 1) * bs], ref, f"c4 final step h{h} ib{ib}")
 
 
-def test_config5_schedule_layers_sampled():
-    """Four layers of projected Q/K/V at 32k with a 16k prompt; the schedule helper drives the mode."""
+@pytest.mark.parametrize("via_stats", [False, True], ids=["two_pass", "from_stats"])
+def test_config5_schedule_layers_sampled(via_stats):
+    """Four layers of projected Q/K/V at 32k with a 16k prompt; the schedule helper drives the mode.
+    The sampled query blocks include the two that straddle the prompt boundary."""
     cfg = syn.CONFIGS["c5"]
     s = sd.sparsed_switch_step(cfg.total_steps, cfg.skip)
     assert s == 64
@@ -170,7 +202,7 @@ def test_config5_schedule_layers_sampled():
     for layer in (0, 3):
         q, k, v = syn.make_qkv(cfg, DEV, layer=layer)
         n_exact, n_rows, worst, (_, _, pat, _, _) = check_sampled(cfg, q, k, v, [1, 17, 30], 4, 50 + layer,
-                                                                  f"c5 layer {layer}")
+                                                                  f"c5 layer {layer}", via_stats=via_stats)
         assert pat.nnz == 32 * 256 * 26
         del q, k, v
         torch.cuda.empty_cache()

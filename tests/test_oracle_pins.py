@@ -285,6 +285,59 @@ def test_sparse_single_kept_block_is_attention_over_that_block():
         np.testing.assert_allclose(o[0, 0, ib * bs:(ib + 1) * bs], sub_o[0, 0], rtol=1e-12, atol=1e-14)
 
 
+def test_batch_two_gqa_and_custom_scale_against_library_routines_and_brute_force():
+    """Row indexing over (batch, head, query block) and the `scale` argument of the full, pooled and
+    masked paths: different data per batch entry, grouped heads, scale 0.37, against torch's SDPA
+    (mask and scale given to the library), torch's avg_pool2d of a library softmax, and the scalar
+    brute force (which knows only 1/sqrt(d): the scale is folded into the queries first)."""
+    B, Hq, Hkv, L, D, bs, scale = 2, 4, 2, 48, 6, 8, 0.37
+    nb, g = L // bs, Hq // Hkv
+    q, k, v = _qkv(B, Hq, Hkv, L, D, 140, qscale=1.4)
+    tq = torch.from_numpy(q)
+    tk = torch.from_numpy(k).repeat_interleave(g, dim=1)
+    tv = torch.from_numpy(v).repeat_interleave(g, dim=1)
+    # Eq. 1 with a custom scale
+    o, lse = orc.attn_full(q, k, v, scale=scale, block_rows=8)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, scale=scale)
+    np.testing.assert_allclose(o, ref.numpy(), rtol=1e-12, atol=1e-13)
+    logits = scale * torch.einsum("bhid,bhjd->bhij", tq, tk)
+    np.testing.assert_allclose(lse, torch.logsumexp(logits, dim=-1).numpy(), rtol=1e-12, atol=1e-13)
+    # avgpool(A): library softmax + library average pooling, every (batch, head)
+    ap = orc.pooled_scores(q, k, bs, scale=scale)
+    pooled_ref = torch.nn.functional.avg_pool2d(torch.softmax(logits, dim=-1).reshape(B * Hq, 1, L, L), bs)
+    np.testing.assert_allclose(ap.reshape(B * Hq, nb, nb), pooled_ref[:, 0].numpy(), rtol=1e-12, atol=1e-16)
+    assert np.abs(ap[0] - ap[1]).max() > 1e-4          # the two batch entries really differ
+    # and the brute force, with the scale folded into q (scale * q.k = (q * scale * sqrt(D)).k / sqrt(D))
+    qf = q * (scale * math.sqrt(D))
+    for b, h in ((0, 1), (1, 0), (1, 3)):
+        np.testing.assert_allclose(ap[b, h], bf.avgpool(bf.score_matrix(qf[b, h], k[b, h // g]), bs),
+                                   rtol=1e-12, atol=1e-15)
+    # Eq. 3 / Eq. 4 with per-(batch, head, block) lists that differ everywhere
+    rp, ci = orc.select_blocks(ap, bs, 24, 0.4)
+    assert rp[-1] == B * Hq * nb * 4
+    o_sp = orc.attn_sparse(q, k, v, rp, ci, bs, scale=scale)
+    mask = torch.zeros(B, Hq, L, L, dtype=torch.bool)
+    lists = {}
+    for b in range(B):
+        for h in range(Hq):
+            for ib in range(nb):
+                r = (b * Hq + h) * nb + ib
+                lists[(b, h, ib)] = list(ci[rp[r]:rp[r + 1]])
+                for jb in lists[(b, h, ib)]:
+                    mask[b, h, ib * bs:(ib + 1) * bs, jb * bs:(jb + 1) * bs] = True
+    assert len({tuple(x) for x in lists.values()}) > 4
+    ref_sp = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=mask, scale=scale)
+    np.testing.assert_allclose(o_sp, ref_sp.numpy(), rtol=1e-12, atol=1e-13)
+    for b, h in ((1, 2), (0, 3)):
+        rows = [lists[(b, h, ib)] for ib in range(nb)]
+        a = bf.score_matrix(qf[b, h], k[b, h // g], bf.token_mask(rows, bs, L))
+        np.testing.assert_allclose(o_sp[b, h], bf.attend(a, v[b, h // g]), rtol=1e-12, atol=1e-13)
+    # head_sparse_rows / head_pooled_row (the per-row-block forms the sampled GPU tests use) agree
+    np.testing.assert_allclose(orc.head_pooled_row(q[1, 2], k[1, 1], 3, bs, scale=scale), ap[1, 2, 3], rtol=1e-13)
+    np.testing.assert_allclose(orc.head_sparse_rows(q[1, 2], k[1, 1], v[1, 1], 3, lists[(1, 2, 3)], bs, scale=scale),
+                               o_sp[1, 2, 3 * bs:4 * bs], rtol=1e-13)
+
+
 # ------------------------------------------------------------------ schedule (Algorithm 1)
 def test_schedule_table():
     for T, skip, s, n_full, n_sparse in _rows("schedule_table.txt"):

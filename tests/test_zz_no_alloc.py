@@ -3,17 +3,23 @@
 Some hosts of this library cannot call cudaMalloc when they need a pattern: a serving process
 that handed all device memory to its own pool at start-up, or a request path where allocation
 is banned because it stalls the device. For them the library carries a fixed scratch array of
-its own. This test calls that entry point through the C ABI twice in a row, with different
-shapes and with and without a caller-supplied LSE, and checks each result against the regular
-entry point (same kernels, so the block lists must be identical), and that oversized requests
-are refused. Collected last on purpose: a failure here must not hide any other test.
+its own. This test calls that entry point through the C ABI several times in a row, with different
+shapes, with and without a caller-supplied LSE, and once with 32-token blocks (the case in which
+the pooled scores and the LSE rows really live in the library's array and are read back from it),
+and checks each result against the regular entry point (same kernels, so the block lists must be
+identical) and against the CPU oracle's selection, and that oversized requests are refused.
+Collected last on purpose: a failure here must not hide any other test.
 """
+import numpy as np
 import pytest
 import torch
 
 import paper_2509_24014_b200 as sd
+from oracle import sparsed_oracle as orc
 from paper_2509_24014_b200 import synthetic as syn
 from paper_2509_24014_b200.binding import STATIC_SCRATCH_BYTES
+from tests.parity_util import to_f64
+from tests.test_gpu_parity_configs import check_row_list
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -46,6 +52,10 @@ def test_static_scratch_selection_matches_regular_entry_point_twice():
         # (config, use the LSE of a full-attention pass?)
         (syn.AttnConfig("a", 1, 4, 2, 2048, 128, 128, 0.25, 1024, seed=21), False),
         (syn.AttnConfig("b", 1, 2, 2, 1024, 128, 64, 0.3, 0, seed=22), True),
+        # 32-token blocks are never ranked inside the scoring kernel: A' and the LSE rows go through the
+        # static array (over what the two calls above left there) and the ranking kernel reads A' back
+        (syn.AttnConfig("c", 1, 2, 2, 1024, 128, 32, 0.5, 512, seed=23), False),
+        (syn.AttnConfig("a", 1, 4, 2, 2048, 128, 128, 0.25, 1024, seed=21), False),
     ]
     for cfg, with_lse in calls:
         q, k, v = syn.make_qkv(cfg, DEV)
@@ -64,6 +74,17 @@ def test_static_scratch_selection_matches_regular_entry_point_twice():
         assert torch.equal(ci_s, ci_r)
         ws = sd.new_workspace(256, DEV)
         assert sd.sparsed_pattern_validate(pat_s, ws)
+        # and against the oracle's own fp64 scores and ranking: list lengths and order exact, every block
+        # clearly above / below the boundary in / out, rows with a clear boundary identical
+        a_ref = orc.pooled_scores(to_f64(q), to_f64(k), cfg.block_size)
+        rp, ci = rp_s.cpu().numpy(), ci_s.cpu().numpy()
+        nb, pb = cfg.num_blocks, cfg.prefill_len // cfg.block_size
+        n_exact = 0
+        for h in range(cfg.heads_q):
+            for ib in range(nb):
+                r = h * nb + ib
+                n_exact += check_row_list(ci[rp[r]:rp[r + 1]], a_ref[0, h, ib], pb, cfg.keep_ratio)
+        assert n_exact > 0     # rows whose boundary gap is wider than the score tolerance matched exactly
 
 
 def test_static_scratch_rejects_requests_beyond_its_size():
