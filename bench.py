@@ -290,7 +290,7 @@ def run_ours(args, cfg):
     shape_qkvo = sd.make_shape(q, k, v, o_full)
     shape_qk = sd.make_shape(q, k)
     ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_PATTERN, shape_qk, params), dev)
-    tile_stats = sd.new_tile_stats(q)
+    tile_stats = sd.new_tile_stats(q, cfg.block_size)
     total_steps, skip = max(cfg.total_steps, 2), (cfg.skip if cfg.total_steps > 1 else 0.5)
     s_switch = sd.sparsed_switch_step(total_steps, skip)
 
@@ -305,7 +305,7 @@ def run_ours(args, cfg):
                 e = ev(); e.record(); marks.append(e)
         mark()
         assert sd.sparsed_schedule_mode(s_switch, total_steps, skip) == sd.MODE_FULL_AND_SELECT
-        sd.sparsed_attn_full_stats(q, k, v, o_full, lse, tile_stats, ws, shape=shape_qkvo)
+        sd.sparsed_attn_full_stats(q, k, v, o_full, lse, tile_stats, ws, cfg.block_size, shape=shape_qkvo)
         mark()
         sd.sparsed_select_from_stats(q, k, params, lse, tile_stats, pat, ws, shape=shape_qk)
         mark()
@@ -571,7 +571,7 @@ def run_schedule_loop(args, cfg, emit=True):
         layers.append({"base": base, "qkv": qkv, "pat": pat, "row_ptr": row_ptr, "col_idx": col_idx})
     o = torch.empty(B, Hq, L, cfg.head_dim, dtype=torch.bfloat16, device=dev)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
-    stats = torch.empty(B * Hq, (L + 63) // 64, L, dtype=torch.float32, device=dev)
+    stats = sd.new_tile_stats(o, bs)
     times = {"full": [], "select": [], "sparse": []}
     sample_heads = [0, Hq // 2, Hq - 1]
     sample_blocks = [0, nb // 2 + 1, nb - 1]
@@ -580,7 +580,7 @@ def run_schedule_loop(args, cfg, emit=True):
     # warm-up of the three kernels
     q, k, v = layers[0]["qkv"] if layers[0]["qkv"] is not None else syn.make_qkv(cfg, dev, 0, step=0, base=layers[0]["base"])
     for _ in range(2):
-        sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+        sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, bs)
         sd.sparsed_select_from_stats(q, k, params, lse, stats, layers[0]["pat"], ws)
         sd.sparsed_attn_sparse(q, k, v, o, layers[0]["pat"], ws)
     torch.cuda.synchronize()
@@ -599,7 +599,7 @@ def run_schedule_loop(args, cfg, emit=True):
                 b.record()
                 times["full"].append((a, b))
             elif mode == sd.MODE_FULL_AND_SELECT:
-                sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+                sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, bs)
                 b.record()
                 sd.sparsed_select_from_stats(q, k, params, lse, stats, lay["pat"], ws)
                 c.record()
@@ -688,7 +688,7 @@ def run_sweep(args, cfg):
     bs, nb = cfg.block_size, cfg.num_blocks
     o = torch.empty_like(q)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
-    stats = sd.new_tile_stats(q)
+    stats = sd.new_tile_stats(q, bs)
     ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_PATTERN, sd.make_shape(q, k),
                                                       sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)), dev)
 
@@ -704,7 +704,7 @@ def run_sweep(args, cfg):
         return statistics.median(ts)
 
     full_ms = timed(lambda: sd.sparsed_attn_full(q, k, v, o, None, ws), reps=3)
-    full_stats_ms = timed(lambda: sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws), reps=3)
+    full_stats_ms = timed(lambda: sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, bs), reps=3)
     rows = []
     for rho in (0.05, 0.1, 0.2, 0.3, 0.5):
         for p_len in sorted({0, cfg.prefill_len, L // 2}):
@@ -765,7 +765,7 @@ def run_estimate_recall(args, cfg):
     k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
     o_full, o_sp = torch.empty_like(q), torch.empty_like(q)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
-    stats = sd.new_tile_stats(q)
+    stats = sd.new_tile_stats(q, bs)
     ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_POOLED_QK, sd.make_shape(q, k), params), dev)
     scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=dev)
     pat_x, rp_x, ci_x = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
@@ -782,7 +782,7 @@ def run_estimate_recall(args, cfg):
             ts.append(a.elapsed_time(b))
         return statistics.median(ts)
 
-    sd.sparsed_attn_full_stats(q, k, v, o_full, lse, stats, ws)
+    sd.sparsed_attn_full_stats(q, k, v, o_full, lse, stats, ws, bs)
     exact_ms = timed(lambda: sd.sparsed_select_from_stats(q, k, params, lse, stats, pat_x, ws, scores_out=scores))
     est_ms = timed(lambda: sd.sparsed_select_pattern_pooled_qk(q, k, params, pat_e, ws))
     torch.cuda.synchronize()

@@ -130,22 +130,27 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
  * step and then computes A' = avgpool(A) from the same Q and K; A' can be formed from row
  * statistics of that very full-attention pass:
  *   sparsed_attn_full_stats   = sparsed_attn_full that also records, for every query row and
- *                               every 64-key tile, log2 of the tile's share of the row's softmax
- *                               denominator (tile_stats, device fp32, sparsed_tile_stats_bytes()
- *                               bytes, layout [batch*heads_q][ceil(seq_len/128)][ceil(seq_len/64)][128]:
- *                               128-row query tile, 64-key tile, row in the query tile);
- *                               lse is required here.
+ *                               every key block of `block_size` keys (32, 64 or 128: the block size
+ *                               the pattern will be selected with), log2 of the block's share of the
+ *                               row's softmax denominator (tile_stats, device fp32,
+ *                               sparsed_tile_stats_bytes() bytes, layout
+ *                               [batch*heads_q][ceil(seq_len/128)][seq_len/block_size][128]:
+ *                               128-row query tile, key block, row in the query tile);
+ *                               lse is required here; seq_len must be a multiple of block_size.
  *   sparsed_select_from_stats = pools those statistics into A' (2^(stat - LSE) is the
- *                               probability mass a row puts on a tile), ranks it as
+ *                               probability mass a row puts on a key block), ranks it as
  *                               sparsed_select_pattern does (Eq. 5 / Eq. 6) and writes the CSR
  *                               pattern; scores_out_or_null optionally receives A'.
+ *                               params->block_size must be the block size the statistics were
+ *                               recorded with.
  * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; the selection needs
- * seq_len <= 131072 and block_size 64 or 128 (the statistics are per 64 keys; UNSUPPORTED otherwise). Both buffers are caller-owned device memory.
+ * seq_len / block_size <= 2048 (UNSUPPORTED beyond). Both buffers are caller-owned device memory.
  */
-sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, size_t *out_bytes); /* host only */
-sparsed_status sparsed_attn_full_stats(const sparsed_shape *shape, const void *q, const void *k, const void *v,
-                                       void *o, float *lse, float *tile_stats, void *ws, size_t ws_bytes,
-                                       void *cuda_stream);
+sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, int32_t block_size,
+                                        size_t *out_bytes); /* host only */
+sparsed_status sparsed_attn_full_stats(const sparsed_shape *shape, int32_t block_size, const void *q,
+                                       const void *k, const void *v, void *o, float *lse, float *tile_stats,
+                                       void *ws, size_t ws_bytes, void *cuda_stream);
 sparsed_status sparsed_select_from_stats(const sparsed_shape *shape, const sparsed_select_params *params,
                                          const float *lse, const float *tile_stats, sparsed_pattern *out,
                                          float *scores_out_or_null, void *ws, size_t ws_bytes, void *cuda_stream);
@@ -175,7 +180,8 @@ sparsed_status sparsed_select_pattern_pooled_qk(const sparsed_shape *shape, cons
  * mask given by `pattern` (Eq. 3 and Eq. 4; the "Sparse Reusing" branch of Algorithm 1).
  * Accepts any CSR whose rows are ascending and in range (not only selected ones); a query
  * block with an empty list gets zeros. Requires seq_len == pattern->num_blocks *
- * pattern->block_size. Errors: as above plus PATTERN.
+ * pattern->block_size; with 64- or 32-key blocks at most 2048 blocks per row (UNSUPPORTED
+ * beyond). Errors: as above plus PATTERN.
  */
 sparsed_status sparsed_attn_sparse(const sparsed_shape *shape, const sparsed_pattern *pattern, const void *q,
                                    const void *k, const void *v, void *o, void *ws, size_t ws_bytes,
@@ -201,12 +207,12 @@ int32_t sparsed_switch_step(int32_t total_steps, double skip);
  *                                   switch step left it ("Sparse Reusing")   -> SPARSED_MODE_SPARSE
  * The same calls as sparsed_attn_full / sparsed_attn_full_stats + sparsed_select_from_stats /
  * sparsed_attn_sparse, chosen by sparsed_schedule_mode; where the statistics path does not apply
- * (block_size 32, seq_len > 131072) the switch step selects with sparsed_select_pattern instead.
+ * (more than 2048 key blocks per row) the switch step selects with sparsed_select_pattern instead.
  * q, k, v, o: device bf16 as for sparsed_attn_full. pattern: caller-owned CSR buffers sized as for
  * sparsed_select_pattern, written at the switch step and only read afterwards; the caller keeps it
  * (one per layer) across steps. ws: device workspace, zeroed status block first; the switch step
  * needs sparsed_workspace_bytes(SPARSED_OP_ATTENTION_STEP, shape, params) bytes (row statistics of
- * the full pass: about 4 * seq_len * ceil(seq_len / 64) bytes per head), every other step only
+ * the full pass: about 4 * seq_len * seq_len / block_size bytes per head), every other step only
  * SPARSED_STATUS_BYTES. mode_out_or_null (host) receives the mode that ran. Errors as for the calls
  * it makes; INVALID_ARG for a step outside 1..total_steps or skip outside [0, 1]. Asynchronous.
  */

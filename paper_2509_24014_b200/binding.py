@@ -86,8 +86,8 @@ def load_library() -> ctypes.CDLL:
     lib.sparsed_select_pattern_static.argtypes = [P(Shape), P(SelectParams), vp, vp, vp, P(Pattern), vp]
     lib.sparsed_build_window_pattern.argtypes = [i32, i32, i32, i32, i32, i32, P(Pattern), vp]
     lib.sparsed_selftest_wait_timeout.argtypes = [vp, sz, vp]
-    lib.sparsed_tile_stats_bytes.argtypes = [P(Shape), P(sz)]
-    lib.sparsed_attn_full_stats.argtypes = [P(Shape), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sparsed_tile_stats_bytes.argtypes = [P(Shape), i32, P(sz)]
+    lib.sparsed_attn_full_stats.argtypes = [P(Shape), i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sparsed_select_from_stats.argtypes = [P(Shape), P(SelectParams), vp, vp, P(Pattern), vp, vp, sz, vp]
     lib.sparsed_select_from_scores.argtypes = [P(SelectParams), vp, i32, i32, i32, P(Pattern), vp, sz, vp]
     lib.sparsed_attn_sparse.argtypes = [P(Shape), P(Pattern), vp, vp, vp, vp, vp, sz, vp]
@@ -254,25 +254,27 @@ def sparsed_attention_step_variant(q, k, v, o, params: SelectParams, variant: in
     return int(mode.value)
 
 
-def sparsed_tile_stats_bytes(shape: Shape) -> int:
+def sparsed_tile_stats_bytes(shape: Shape, block_size: int) -> int:
     out = ctypes.c_size_t()
-    _check(load_library().sparsed_tile_stats_bytes(ctypes.byref(shape), ctypes.byref(out)), "sparsed_tile_stats_bytes")
+    _check(load_library().sparsed_tile_stats_bytes(ctypes.byref(shape), int(block_size), ctypes.byref(out)),
+           "sparsed_tile_stats_bytes")
     return int(out.value)
 
 
-def new_tile_stats(q: torch.Tensor) -> torch.Tensor:
-    """Caller-owned buffer for sparsed_attn_full_stats: fp32 [B*Hq, ceil(L/128), ceil(L/64), 128]."""
+def new_tile_stats(q: torch.Tensor, block_size: int) -> torch.Tensor:
+    """Caller-owned buffer for sparsed_attn_full_stats: fp32 [B*Hq, ceil(L/128), L/block_size, 128]."""
     B, Hq, L, _ = q.shape
-    return torch.empty(B * Hq, (L + 127) // 128, (L + 63) // 64, 128, dtype=torch.float32, device=q.device)
+    return torch.empty(B * Hq, (L + 127) // 128, L // block_size, 128, dtype=torch.float32, device=q.device)
 
 
 def sparsed_attn_full_stats(q, k, v, o, lse: torch.Tensor, tile_stats: torch.Tensor, ws: torch.Tensor,
-                            softmax_scale: float = 0.0, shape: Optional[Shape] = None) -> None:
+                            block_size: int, softmax_scale: float = 0.0, shape: Optional[Shape] = None) -> None:
+    """block_size: the pattern block size the statistics are recorded for (one statistic per row and key block)."""
     shape = shape or make_shape(q, k, v, o, softmax_scale)
-    assert tile_stats.numel() * 4 >= sparsed_tile_stats_bytes(shape) and tile_stats.dtype == torch.float32
-    _check(load_library().sparsed_attn_full_stats(ctypes.byref(shape), q.data_ptr(), k.data_ptr(), v.data_ptr(),
-                                                  o.data_ptr(), lse.data_ptr(), tile_stats.data_ptr(), ws.data_ptr(),
-                                                  ws.numel(), _stream(q)), "sparsed_attn_full_stats")
+    assert tile_stats.numel() * 4 >= sparsed_tile_stats_bytes(shape, block_size) and tile_stats.dtype == torch.float32
+    _check(load_library().sparsed_attn_full_stats(ctypes.byref(shape), int(block_size), q.data_ptr(), k.data_ptr(),
+                                                  v.data_ptr(), o.data_ptr(), lse.data_ptr(), tile_stats.data_ptr(),
+                                                  ws.data_ptr(), ws.numel(), _stream(q)), "sparsed_attn_full_stats")
 
 
 def sparsed_select_from_stats(q, k, params: SelectParams, lse: torch.Tensor, tile_stats: torch.Tensor,

@@ -188,7 +188,7 @@ size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Whether the switch step can select from the row statistics of its own full-attention pass.
 bool step_uses_stats(const sparsed_shape* shape, const sparsed_select_params* params) {
-  return params->block_size != 32 && shape->seq_len <= 131072;
+  return shape->seq_len / params->block_size <= pool_select_max_blocks();
 }
 
 // Checks the caller's pattern buffers against the number of rows and kept blocks per row and
@@ -317,7 +317,7 @@ sparsed_status sparsed_workspace_bytes(int32_t op, const sparsed_shape* shape, c
       const size_t lse_bytes = round_up(bh * static_cast<size_t>(shape->seq_len) * 4, 256);
       if (step_uses_stats(shape, params)) {
         size_t stats = 0;
-        sparsed_status st = sparsed_tile_stats_bytes(shape, &stats);
+        sparsed_status st = sparsed_tile_stats_bytes(shape, params->block_size, &stats);
         if (st != SPARSED_OK) return st;
         *out_bytes = SPARSED_STATUS_BYTES + lse_bytes + stats;
       } else {
@@ -338,8 +338,8 @@ sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stre
 }
 
 static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
-                                     float* lse_or_null, float* tile_lse_or_null, void* ws, size_t ws_bytes,
-                                     void* cuda_stream) {
+                                     float* lse_or_null, float* tile_lse_or_null, int stat_keys, void* ws,
+                                     size_t ws_bytes, void* cuda_stream) {
   Resolved rs;
   sparsed_status st = check_shape(shape, true, &rs);
   if (st != SPARSED_OK) return st;
@@ -360,12 +360,13 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   p.o_stride_t = rs.o[2];
   p.lse = lse_or_null;
   p.tile_lse = tile_lse_or_null;
-  p.stat_keys = 64;
+  p.stat_keys = stat_keys;
   p.slow_path_events = reinterpret_cast<unsigned long long*>(static_cast<uint8_t*>(ws) + 32);
   p.seq_len = shape->seq_len;
   p.heads_q = shape->heads_q;
   p.group = shape->heads_q / shape->heads_kv;
   p.num_q_tiles = (shape->seq_len + 127) / 128;
+  p.num_blocks = 0;
   p.scale_log2 = rs.scale_log2;
   p.row_ptr = nullptr;
   p.col_idx = nullptr;
@@ -376,23 +377,27 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
 
 sparsed_status sparsed_attn_full(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
                                  float* lse_or_null, void* ws, size_t ws_bytes, void* cuda_stream) {
-  return attn_full_impl(shape, q, k, v, o, lse_or_null, nullptr, ws, ws_bytes, cuda_stream);
+  return attn_full_impl(shape, q, k, v, o, lse_or_null, nullptr, 64, ws, ws_bytes, cuda_stream);
 }
 
-sparsed_status sparsed_tile_stats_bytes(const sparsed_shape* shape, size_t* out_bytes) {
+sparsed_status sparsed_tile_stats_bytes(const sparsed_shape* shape, int32_t block_size, size_t* out_bytes) {
   if (shape == nullptr || out_bytes == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (shape->batch < 1 || shape->heads_q < 1 || shape->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
-  const size_t tiles = (static_cast<size_t>(shape->seq_len) + 63) / 64;
+  if (block_size != 32 && block_size != 64 && block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (shape->seq_len % block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  const size_t groups = static_cast<size_t>(shape->seq_len / block_size);
   const size_t q_tiles = (static_cast<size_t>(shape->seq_len) + 127) / 128;
-  *out_bytes = static_cast<size_t>(shape->batch) * shape->heads_q * q_tiles * tiles * 128 * 4;
+  *out_bytes = static_cast<size_t>(shape->batch) * shape->heads_q * q_tiles * groups * 128 * 4;
   return SPARSED_OK;
 }
 
-sparsed_status sparsed_attn_full_stats(const sparsed_shape* shape, const void* q, const void* k, const void* v,
-                                       void* o, float* lse, float* tile_stats, void* ws, size_t ws_bytes,
-                                       void* cuda_stream) {
-  if (lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
-  return attn_full_impl(shape, q, k, v, o, lse, tile_stats, ws, ws_bytes, cuda_stream);
+sparsed_status sparsed_attn_full_stats(const sparsed_shape* shape, int32_t block_size, const void* q, const void* k,
+                                       const void* v, void* o, float* lse, float* tile_stats, void* ws,
+                                       size_t ws_bytes, void* cuda_stream) {
+  if (shape == nullptr || lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
+  if (block_size != 32 && block_size != 64 && block_size != 128) return SPARSED_ERR_UNSUPPORTED;
+  if (shape->seq_len >= 1 && shape->seq_len % block_size != 0) return SPARSED_ERR_ALIGNMENT;
+  return attn_full_impl(shape, q, k, v, o, lse, tile_stats, block_size, ws, ws_bytes, cuda_stream);
 }
 
 sparsed_status sparsed_select_from_stats(const sparsed_shape* shape, const sparsed_select_params* params,
@@ -408,8 +413,7 @@ sparsed_status sparsed_select_from_stats(const sparsed_shape* shape, const spars
   if (st != SPARSED_OK) return st;
   if (lse == nullptr || tile_stats == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (!aligned16(lse) || !aligned16(tile_stats) || !aligned16(scores_out_or_null)) return SPARSED_ERR_ALIGNMENT;
-  // the recorded statistics are per 64 keys: 32-key blocks need sparsed_select_pattern
-  if (shape->seq_len > 131072 || params->block_size == 32) return SPARSED_ERR_UNSUPPORTED;
+  if (nb > pool_select_max_blocks()) return SPARSED_ERR_UNSUPPORTED;
   if ((st = prepare_pattern(out, shape->batch, shape->heads_q, nb, params->block_size, k_pre + k_gen)) != SPARSED_OK)
     return st;
   if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
@@ -495,8 +499,9 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
   const int bs = pattern->block_size;
+  if (pattern->num_blocks > attn_sparse_max_blocks(bs)) return SPARSED_ERR_UNSUPPORTED;
   CUtensorMap tq, tk, tv;
-  if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, bs)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
   const int kv_box = bs < 64 ? bs : 64;
   if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, kv_box)) != SPARSED_OK) return st;
   if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, kv_box)) != SPARSED_OK) return st;
@@ -512,7 +517,8 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   p.seq_len = shape->seq_len;
   p.heads_q = shape->heads_q;
   p.group = shape->heads_q / shape->heads_kv;
-  p.num_q_tiles = pattern->num_blocks;
+  p.num_q_tiles = (shape->seq_len + 127) / 128;
+  p.num_blocks = pattern->num_blocks;
   p.scale_log2 = rs.scale_log2;
   p.row_ptr = pattern->row_ptr;
   p.col_idx = pattern->col_idx;
@@ -621,7 +627,8 @@ sparsed_status sparsed_attention_step(const sparsed_shape* shape, const sparsed_
   if (step_uses_stats(shape, params)) {
     float* lse = reinterpret_cast<float*>(base + SPARSED_STATUS_BYTES);
     float* stats = reinterpret_cast<float*>(base + SPARSED_STATUS_BYTES + lse_bytes);
-    if ((st = sparsed_attn_full_stats(shape, q, k, v, o, lse, stats, ws, ws_bytes, cuda_stream)) != SPARSED_OK) return st;
+    if ((st = sparsed_attn_full_stats(shape, params->block_size, q, k, v, o, lse, stats, ws, ws_bytes, cuda_stream)) != SPARSED_OK)
+      return st;
     return sparsed_select_from_stats(shape, params, lse, stats, pattern, nullptr, ws, ws_bytes, cuda_stream);
   }
   // [status][A' scratch of sparsed_select_pattern][LSE of the full pass]

@@ -2,10 +2,10 @@
 // head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a. (Dense attention has its own
 // two-tiles-per-CTA kernel in attention_dense.cu.)
 //
-// One CTA owns one query tile of one (batch, head) and streams 64-key tiles through a
+// One CTA owns 128 consecutive query rows of one (batch, head) and streams 64-key tiles through a
 // warp-specialised pipeline:
-//   warp 4  : TMA producer  - Q once, then a K tile and a V tile per step into a five-slot
-//                             ring of 128B-swizzled shared memory shared by K and V
+//   warp 4  : TMA producer  - Q once, then a K tile and a V tile per step into a ring of
+//                             128B-swizzled shared memory shared by K and V
 //   warp 5  : UMMA issuer   - S_j = Q K_j^T into one of two tensor-memory buffers, then
 //                             O += P_j V_j with P read from tensor memory (P overwrites the
 //                             first half of S_j's columns). S_{j+1} is issued before P_j V_j,
@@ -15,14 +15,20 @@
 //                             softmax warps "S_j is ready" / "P_j V_j has drained" and the producer
 //                             "the slot is free" (the issuing thread is the pipeline's bottleneck:
 //                             a commit costs it about 150 clocks, a barrier poll about 100).
-//   warps 0-3: one thread per query row - online softmax in fp32 on base-2 logits. The tile
-//             is exponentiated once against the running maximum; only if a row sum shows that
-//             logits may have outgrown it by more than 2^8 is the tile redone with the new
-//             maximum and O rescaled (after the previous P V has drained). Finally O is
-//             normalised and stored.
-// The tile index comes from the CSR list of the CTA's query block (a 128-key block is two
-// consecutive tiles, two 32-key blocks share one). Two CTAs fit on one SM (112 KB of shared memory
-// and 256 tensor-memory columns each).
+//   warps 0-3: one thread per query row - single-pass online softmax in fp32 on base-2 logits
+//             against a stale running maximum (softmax_pipeline.cuh); finally O is normalised
+//             and stored.
+// Two CTAs fit on one SM (at most 112 KB of shared memory and 256 tensor-memory columns each).
+//
+// Where the keys come from:
+//   * 128-key blocks: the 128 query rows are one query block; its CSR list is walked as it is,
+//     two tiles per block.
+//   * 64- and 32-key blocks: the 128 query rows are two / four consecutive query blocks with lists
+//     of their own. The CTA walks the UNION of those lists (built in shared memory at start-up as one
+//     bitmap per query block) and every warp masks, per 32-column chunk of a tile, the key blocks
+//     its own query block did not keep; a tile in which a warp keeps nothing costs it no
+//     exponentials. All 128 rows of every MMA belong to real queries, and neighbouring query blocks
+//     share the K/V tiles they have in common.
 #include "internal.h"
 #include "softmax_pipeline.cuh"
 
@@ -32,12 +38,12 @@ namespace {
 constexpr int kHeadDim = 128;
 constexpr int kTileM = 128;   // UMMA M; rows of tensor memory
 constexpr int kTileN = 64;    // keys per pipeline step
-constexpr int kSlots = 5;     // ring of 64-key tiles shared by K and V: load 2t is K_t, load 2t+1 is V_t
 constexpr int kSoftmaxThreads = 128;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0;      // two S buffers of 64 fp32 columns; P (bf16 pairs) reuses the first 32
 constexpr int kColO = 128;    // O accumulator (fp32, 128 columns)
+constexpr int kMaxPackedBlocks = 2048;   // key blocks per row the union walk can hold (64- and 32-key blocks)
 #ifndef SPARSED_ATTN_POLY_EVERY
 #define SPARSED_ATTN_POLY_EVERY 0
 #endif
@@ -46,14 +52,20 @@ constexpr int kPolyEvery = SPARSED_ATTN_POLY_EVERY;  // every n-th exponential o
 // Debug builds (-DSPARSED_TIMELINE) record clock64 stamps of one CTA's pipeline roles after the
 // workspace status block: 3 regions of 2048 int64 (softmax thread 0, UMMA thread, TMA thread).
 #ifdef SPARSED_TIMELINE
-#define TL_DECL(region) long long* tl_buf = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(p.status) + 1024) + (region) * 2048; int tl_n = 0; const bool tl_on = (blockIdx.x == 1000) && ((threadIdx.x & 31) == 0);
+#define TL_DECL(region) long long* tl_buf = reinterpret_cast<long long*>(reinterpret_cast<uint8_t*>(p.status) + 1024) + (region) * 2048; int tl_n = 0; const bool tl_on = (blockIdx.x == 1000) && (threadIdx.x == 0 || threadIdx.x == 128 || threadIdx.x == 160);
 #define TL(tag) do { if (tl_on && tl_n < 2047) { tl_buf[1 + tl_n++] = (static_cast<long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFll); tl_buf[0] = tl_n; } } while (0)
 #else
 #define TL_DECL(region)
 #define TL(tag)
 #endif
 
+// Ring slots: five for 128-key blocks; four when the union walk needs room for its lists.
+template <int kBlock>
 struct AttnSmem {
+  static constexpr bool kPacked = kBlock < kTileM;
+  static constexpr int kSlots = kPacked ? 4 : 5;
+  static constexpr int kGroups = kTileM / kBlock;                       // query blocks per CTA
+  static constexpr int kWords = kPacked ? kMaxPackedBlocks / 32 : 1;    // bitmap words per query block
   alignas(1024) __nv_bfloat16 q[2][kTileM * 64];           // two 64-wide halves of head_dim
   alignas(1024) __nv_bfloat16 kv[kSlots][2][kTileN * 64];  // each slot: two 64-wide halves of head_dim
   uint64_t q_full, kv_full[kSlots];
@@ -61,16 +73,23 @@ struct AttnSmem {
   uint64_t p_full[2];
   uint32_t tmem_base;
   int abort_flag;
+  int n_union;                                             // packed: key blocks in the union list
+  uint32_t member[kGroups][kWords];                        // packed: bit j of query block g = "g keeps key block j"
+  uint16_t union_ids[kPacked ? kMaxPackedBlocks : 2];      // packed: the union, ascending
 };
 
-// kBlock : keys per pattern block.
-// kRowsQ : valid query rows per tile (32, 64 or 128; the UMMA tile is always 128 rows).
-template <int kBlock, int kRowsQ>
+template <int kBlock>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+  using Smem = AttnSmem<kBlock>;
+  constexpr bool kPacked = Smem::kPacked;
+  constexpr int kSlots = Smem::kSlots;
+  constexpr int kGroups = Smem::kGroups;
+  constexpr int kTilesPerBlock = kBlock >= kTileN ? kBlock / kTileN : 1;   // 128-key block: two tiles
+  constexpr int kBlocksPerTile = kBlock >= kTileN ? 1 : kTileN / kBlock;   // 32-key blocks: two per tile
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  AttnSmem& sm = *reinterpret_cast<AttnSmem*>(smem_raw);
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0u) {
     // swizzled tiles need a 1024-byte aligned base; never expected, reported instead of trusted
     if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, 2) == 0) p.status->where = 1;
@@ -79,44 +98,43 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
-  constexpr int kTilesPerBlock = kBlock >= kTileN ? kBlock / kTileN : 1;   // 128-key block: two tiles
-  constexpr int kBlocksPerTile = kBlock >= kTileN ? 1 : kTileN / kBlock;   // 32-key blocks: two per tile
+  const int lane = tid & 31;
 
   // ---- work item -----------------------------------------------------------------------
+  // num_q_tiles = 128-row query tiles per (batch, head); num_blocks = pattern blocks per row
   const int q_tile = blockIdx.x % p.num_q_tiles;
   const int bh = blockIdx.x / p.num_q_tiles;
   const int head = bh % p.heads_q;
   const int batch = bh / p.heads_q;
   const int kv_head = head / p.group;
-  const int q_row0 = q_tile * kRowsQ;
+  const int q_row0 = q_tile * kTileM;
+  const int qb0 = q_tile * kGroups;                          // first query block of this CTA
+  const int groups_here = min(kGroups, p.num_blocks - qb0);  // the last CTA of a head may hold fewer
+  const int r0 = bh * p.num_blocks + qb0;                    // CSR row of query block qb0
 
-  const int r = bh * p.num_q_tiles + q_tile;
-  const int list_begin = __ldg(p.row_ptr + r);
-  const int list_len = __ldg(p.row_ptr + r + 1) - list_begin;
-  const int num_tiles =
-      kBlocksPerTile == 1 ? list_len * kTilesPerBlock : (list_len + kBlocksPerTile - 1) / kBlocksPerTile;
+  // list_begin / list_len: the CSR entries of this CTA's query blocks (adjacent rows are adjacent in col_idx)
+  const int list_begin = __ldg(p.row_ptr + r0);
+  const int list_len = __ldg(p.row_ptr + r0 + groups_here) - list_begin;
 
   // ---- set-up --------------------------------------------------------------------------
-  // The producer warp starts the two loads nothing else depends on before the CTA-wide set-up has
-  // finished: the Q tile (through a barrier it initialises itself) and the first 32 ids of the list.
-  int list_ids = 0;  // warp 4: lane i holds col_idx[list_begin + 32 * chunk + i] of the current chunk
+  // The producer warp starts the load nothing else depends on before the CTA-wide set-up has
+  // finished: the Q tile, through a barrier it initialises itself.
   if (warp == 4) {
-    if ((tid & 31) == 0) {
+    if (lane == 0) {
       mbar_init(&sm.q_full, 1);
       mbar_fence_init();
     }
     __syncwarp();
-    if (num_tiles > 0) {
+    if (list_len > 0) {
       if (elect_one_sync()) {
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
-        mbar_expect_tx(&sm.q_full, kRowsQ * kHeadDim * 2);
+        mbar_expect_tx(&sm.q_full, kTileM * kHeadDim * 2);   // rows beyond the sequence arrive as zeros
         tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
         tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
       }
       __syncwarp();
-      if ((tid & 31) < list_len) list_ids = __ldg(p.col_idx + list_begin + (tid & 31));
     }
   }
   if (tid == 0) {
@@ -126,21 +144,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     for (int s = 0; s < 2; ++s) mbar_init(&sm.p_full[s], kSoftmaxThreads);
     sm.abort_flag = 0;
+    sm.n_union = 0;
     mbar_fence_init();
   }
-  if constexpr (kRowsQ < kTileM) {
-    // rows the TMA box does not cover are multiplied too: keep them finite (zero)
-    uint4* z0 = reinterpret_cast<uint4*>(&sm.q[0][kRowsQ * 64]);
-    uint4* z1 = reinterpret_cast<uint4*>(&sm.q[1][kRowsQ * 64]);
-    constexpr int n16 = (kTileM - kRowsQ) * 64 * 2 / 16;
-    for (int i = tid; i < n16; i += kThreads) {
-      z0[i] = make_uint4(0, 0, 0, 0);
-      z1[i] = make_uint4(0, 0, 0, 0);
-    }
-    fence_proxy_async_smem();
-  }
   if constexpr (kBlocksPerTile > 1) {
-    // a tile may be half filled (odd list): its other half is multiplied by P = 0, so it has to
+    // a tile may be half filled (odd union): its other half is multiplied by P = 0, so it has to
     // hold finite numbers from the start
     uint4* z = reinterpret_cast<uint4*>(&sm.kv[0][0][0]);
     constexpr int n16 = kSlots * 2 * kTileN * 64 * 2 / 16;
@@ -151,34 +159,83 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     tmem_alloc(&sm.tmem_base, kTmemCols);
     tmem_relinquish();
   }
+  if constexpr (kPacked) {
+    // One bitmap per query block, then their union as an ascending list.
+    const int words = (p.num_blocks + 31) >> 5;
+    for (int i = tid; i < kGroups * Smem::kWords; i += kThreads) (&sm.member[0][0])[i] = 0u;
+    __syncthreads();
+    int bound[kGroups];   // bound[g] = first CSR entry after query block g's list
+#pragma unroll
+    for (int g = 0; g < kGroups; ++g) bound[g] = __ldg(p.row_ptr + r0 + min(g + 1, groups_here));
+    for (int e = list_begin + tid; e < list_begin + list_len; e += kThreads) {
+      const int id = __ldg(p.col_idx + e);
+      int g = 0;
+#pragma unroll
+      for (int j = 0; j + 1 < kGroups; ++j) g += (e >= bound[j]) ? 1 : 0;
+      if (id >= 0 && id < p.num_blocks) atomicOr(&sm.member[g][id >> 5], 1u << (id & 31));
+    }
+    __syncthreads();
+    if (warp == 4) {
+      int base = 0;
+      for (int w0 = 0; w0 < words; w0 += 32) {
+        const int w = w0 + lane;
+        uint32_t bits = 0u;
+        if (w < words) {
+#pragma unroll
+          for (int g = 0; g < kGroups; ++g) bits |= sm.member[g][w];
+        }
+        const int cnt = __popc(bits);
+        int incl = cnt;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, off);
+          if (lane >= off) incl += v;
+        }
+        int pos = base + incl - cnt;
+        while (bits != 0u) {
+          const int b = __ffs(bits) - 1;
+          sm.union_ids[pos++] = static_cast<uint16_t>(w * 32 + b);
+          bits &= bits - 1u;
+        }
+        base += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) sm.n_union = base;
+    }
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   const uint32_t tO = tmem + kColO;
+  const int n_entries = kPacked ? sm.n_union : list_len;   // key blocks this CTA walks
+  const int num_tiles =
+      kBlocksPerTile == 1 ? n_entries * kTilesPerBlock : (n_entries + kBlocksPerTile - 1) / kBlocksPerTile;
 
   // Warps 4 and 5 run their loops with all 32 lanes converged and let one elected lane issue
   // the TMA / UMMA instructions: their operands then stay on the uniform datapath.
   if (warp == 4) {
     // =============================== TMA producer =======================================
     if (num_tiles > 0) {
-      const int lane = tid & 31;
       TL_DECL(2)
       bool ok = true;
+      // unpacked walk: block ids are fetched 32 at a time, one per lane
+      int list_ids = 0;
+      if constexpr (!kPacked) {
+        if (lane < n_entries) list_ids = __ldg(p.col_idx + list_begin + lane);
+      }
       for (int t = 0; ok && t < num_tiles; ++t) {
-        // list entry of this tile's (first) block; ids are fetched 32 at a time, one per lane
+        // entry of this tile's (first) block in the walked list
         const int e = kBlocksPerTile == 1 ? t / kTilesPerBlock : kBlocksPerTile * t;
-        if (e > 0 && (e & 31) == 0 && (kBlocksPerTile > 1 || t % kTilesPerBlock == 0))
-          list_ids = (e + lane < list_len) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
         int kv_row0, kv_row1 = 0, blocks_here = 1;
-        if constexpr (kBlocksPerTile == 1) {
+        if constexpr (!kPacked) {
+          if (e > 0 && (e & 31) == 0 && t % kTilesPerBlock == 0)
+            list_ids = (e + lane < n_entries) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
           kv_row0 = __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock + (t % kTilesPerBlock) * kTileN;
         } else {
-          // two 32-key blocks side by side in one 64-key tile; an odd list leaves the last tile half filled
-          kv_row0 = __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock;
-          const int second = __shfl_sync(0xffffffffu, list_ids, (e + 1) & 31);
-          if (e + 1 < list_len) {
-            kv_row1 = second * kBlock;
+          kv_row0 = static_cast<int>(sm.union_ids[e]) * kBlock;
+          if (kBlocksPerTile > 1 && e + 1 < n_entries) {
+            // two 32-key blocks side by side in one 64-key tile; an odd union leaves the last tile half filled
+            kv_row1 = static_cast<int>(sm.union_ids[e + 1]) * kBlock;
             blocks_here = 2;
           }
         }
@@ -260,13 +317,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     // =============================== softmax / epilogue =================================
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     const float scale_log2 = p.scale_log2;
+    // packed walk: this warp's 32 rows belong to one query block
+    const int my_group = kPacked ? (warp * 32) / kBlock : 0;
+    const bool group_valid = my_group < groups_here;
     bool ok = true;
     TL_DECL(0)
-#ifdef SPARSED_TIMELINE
-    const bool tl_on2 = tl_on && tid == 0;
-#undef TL
-#define TL(tag) do { if (tl_on2 && tl_n < 2047) { tl_buf[1 + tl_n++] = (static_cast<long long>(tag) << 48) | (clock64() & 0xFFFFFFFFFFFFll); tl_buf[0] = tl_n; } } while (0)
-#endif
     RowState st{-INFINITY, 0.f};
     for (int t = 0; t < num_tiles; ++t) {
       TL(1);
@@ -278,35 +333,65 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       TL(2);
       tc_fence_after();
       const uint32_t tS = tmem + kColS + (t & 1) * kTileN + lane_base;
-      uint32_t r0[32], r1[32];
-      tmem_ld32(tS, r0);
-      tmem_ld32(tS + 32, r1);
-      tmem_wait_ld();
-      TL(3);
-      if constexpr (kBlocksPerTile > 1) {
-        // only the last tile can be ragged: an odd block list leaves its second half empty
-        const int valid_cols = (list_len - kBlocksPerTile * t) * kBlock;
-        if (valid_cols < kTileN) mask_columns_from(r0, r1, valid_cols);
-      }
-      uint32_t pk[32];
-      float2 sums = softmax_group_fast<kPolyEvery>(r0, r1, scale_log2, st.m, pk);
-      const bool trigger = !(sums.x + sums.y <= 256.0f);  // also true on the first tile (m = -inf) and for NaN
-      if (__any_sync(0xffffffffu, trigger)) {
-        // first tile, or logits that outgrew the running maximum
-        const float alpha = softmax_group_exact(r0, r1, scale_log2, st, pk, sums);
-        if (t > 0) {
-          // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring slot 2t-1) has drained
-          const int ip = 2 * (t - 1) + 1;
-          if (!mbar_wait(&sm.done[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
-            ok = false;
-            break;
+      // packed walk: which 32-column chunks of this tile hold key blocks this warp's query block kept
+      bool keep0 = true, keep1 = true;
+      if constexpr (kPacked) {
+        const int e = kBlocksPerTile * t;
+        const int id0 = sm.union_ids[e];
+        keep0 = group_valid && ((sm.member[my_group][id0 >> 5] >> (id0 & 31)) & 1u) != 0u;
+        if constexpr (kBlocksPerTile == 1) {
+          keep1 = keep0;
+        } else {
+          keep1 = false;
+          if (e + 1 < n_entries) {
+            const int id1 = sm.union_ids[e + 1];
+            keep1 = group_valid && ((sm.member[my_group][id1 >> 5] >> (id1 & 31)) & 1u) != 0u;
           }
-          tc_fence_after();
-          rescale_accumulator_row(tO + lane_base, alpha);
-          if (p.slow_path_events != nullptr && (tid & 31) == 0) atomicAdd(p.slow_path_events, 1ull);
         }
       }
-      st.l += sums.x + sums.y;
+      uint32_t pk[32];
+      if (kPacked && !keep0 && !keep1) {
+        // nothing of this tile is kept by this warp's query block: P = 0, no exponentials
+#pragma unroll
+        for (int j = 0; j < 32; ++j) pk[j] = 0u;
+      } else {
+        uint32_t r0[32], r1[32];
+        tmem_ld32(tS, r0);
+        tmem_ld32(tS + 32, r1);
+        tmem_wait_ld();
+        TL(3);
+        if constexpr (kPacked) {
+          if (!keep0) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r0[j] = 0xff800000u;   // -inf
+          }
+          if (!keep1) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r1[j] = 0xff800000u;
+          }
+        }
+        float2 sums;
+        bool exact = (st.m == -INFINITY);   // nothing accumulated yet: no reference maximum to try
+        if (!__all_sync(0xffffffffu, exact)) {
+          sums = softmax_group_fast<kPolyEvery>(r0, r1, scale_log2, st.m, pk);
+          exact = !(sums.x + sums.y <= 256.0f);   // logits outgrew the running maximum (or NaN)
+        }
+        if (__any_sync(0xffffffffu, exact)) {
+          const float alpha = softmax_group_exact(r0, r1, scale_log2, st, pk, sums);
+          if (t > 0) {
+            // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring slot 2t-1) has drained
+            const int ip = 2 * (t - 1) + 1;
+            if (!mbar_wait(&sm.done[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            rescale_accumulator_row(tO + lane_base, alpha);
+            if (p.slow_path_events != nullptr && lane == 0) atomicAdd(p.slow_path_events, 1ull);
+          }
+        }
+        st.l += sums.x + sums.y;
+      }
       TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();
@@ -321,10 +406,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       ok = mbar_wait(&sm.done[il % kSlots], (il / kSlots) & 1, &sm.abort_flag, p.status, 31);
     }
     tc_fence_after();
-    const int row_in_tile = tid;
-    const int row = q_row0 + row_in_tile;
-    const bool row_valid = (row_in_tile < kRowsQ) && (row < p.seq_len);
-    const float inv_l = (num_tiles > 0) ? (1.f / st.l) : 0.f;
+    const int row = q_row0 + tid;
+    const bool row_valid = row < p.seq_len;
+    const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
     __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + batch * p.o_stride_b + head * p.o_stride_h +
                            static_cast<int64_t>(row) * p.o_stride_t;
     store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
@@ -339,11 +423,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int kBlock, int kRowsQ>
+template <int kBlock>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kBlock, kRowsQ>;
-  const int smem = static_cast<int>(sizeof(AttnSmem));
+  auto kernel = attn_kernel<kBlock>;
+  const int smem = static_cast<int>(sizeof(AttnSmem<kBlock>));
   static SmemLimit limit;  // per template instantiation
   cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
   if (e != cudaSuccess) return e;
@@ -355,12 +439,15 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
 
 }  // namespace
 
-// Tensor maps: Q box 64 x block_size rows, K and V boxes 64 x min(64, block_size) rows.
+int attn_sparse_max_blocks(int block_size) { return block_size < kTileM ? kMaxPackedBlocks : 16384; }
+
+// Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x min(64, block_size) rows.
+// p.num_q_tiles = ceil(seq_len / 128), p.num_blocks = seq_len / block_size.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128, 128>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<64, 64>(tq, tk, tv, p, batch, stream);
-  return launch<32, 32>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<128>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<64>(tq, tk, tv, p, batch, stream);
+  return launch<32>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed

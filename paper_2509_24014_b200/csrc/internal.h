@@ -45,7 +45,8 @@ struct AttnParams {
   int seq_len;
   int heads_q;
   int group;               // heads_q / heads_kv
-  int num_q_tiles;         // query tiles per (batch, head)
+  int num_q_tiles;         // 128-row query tiles per (batch, head)
+  int num_blocks;          // sparse only: pattern blocks per row (seq_len / block_size)
   float scale_log2;        // softmax scale * log2(e)
   const int32_t* row_ptr;  // sparse only
   const int32_t* col_idx;  // sparse only
@@ -73,13 +74,13 @@ constexpr int kFusedTopkMaxBlocks = 1024;
 
 // Parameters of the kernel that pools per-tile row statistics into A' and ranks it.
 struct PoolParams {
-  const float* tile_lse;   // fp32 [B*Hq, ceil(L/128), tiles, 128], base-2
+  const float* tile_lse;   // fp32 [B*Hq, ceil(L/128), L/block_size, 128], base-2
   const float* lse;        // fp32 [B,Hq,L], natural log
   float* scores;           // fp32 [B,Hq,nb,nb] or null
   int32_t* row_ptr;
   int32_t* col_idx;
   int seq_len;
-  int block_size;          // 64 or 128
+  int block_size;          // 32, 64 or 128 (= keys per statistic)
   int pb, k_pre, k_gen;
   int bh;                  // B * Hq
 };
@@ -117,6 +118,7 @@ size_t pooled_qk_means_bytes(int batch, int heads_q, int heads_kv, int nb);
 cudaError_t launch_pooled_qk_select(const PooledQkParams& p, cudaStream_t stream);
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream);
+int attn_sparse_max_blocks(int block_size);   // most key blocks per row the sparse kernel handles
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream);
 cudaError_t launch_row_stats(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, float* lse_out,
@@ -124,6 +126,7 @@ cudaError_t launch_row_stats(const CUtensorMap& tq, const CUtensorMap& tk, const
 cudaError_t launch_pooled_scores(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int batch,
                                  cudaStream_t stream);
 cudaError_t launch_topk_csr(const TopkParams& p, cudaStream_t stream);
+int pool_select_max_blocks();   // most key blocks per row the statistics path handles
 cudaError_t launch_pool_select(const PoolParams& p, cudaStream_t stream);
 int64_t window_pattern_nnz_per_head(int nb, int sink, int half);
 cudaError_t launch_window_pattern(int32_t* row_ptr, int32_t* col_idx, int bh, int nb, int sink, int half,

@@ -2,21 +2,22 @@
 // ("Isolated Selection": A' = avgpool(A, block_size), then Eq. 5 / Eq. 6), without a second
 // Q K^T pass.
 //
-// The dense attention kernel can record, for every query row i and every 64-key tile t,
-// v[t][i] = log2 sum_{j in t} 2^(s_ij), the tile's share of the row's softmax denominator.
-// With the row's final log-sum-exp, 2^(v[t][i] - LSE_i) is exactly the probability mass row i
-// puts on tile t, so A'[ib][jb] is the sum of that mass over the rows of block ib and the tiles
-// of block jb, divided by block_size^2.
+// The dense attention kernel can record, for every query row i and every group g of block_size
+// keys, v[g][i] = log2 sum_{j in g} 2^(s_ij), the group's share of the row's softmax denominator.
+// With the row's final log-sum-exp, 2^(v[g][i] - LSE_i) is exactly the probability mass row i
+// puts on key block g, so A'[ib][jb] is the sum of that mass over the rows of query block ib,
+// divided by block_size^2.
 //
-// One CTA owns one 128-row query tile of one (batch, head). Statistics are read with 16-byte
-// loads (four consecutive rows of one tile; the layout [bh][128-row query tile][key tile][row]
-// makes a CTA's reads one contiguous run), eight in flight per thread and six CTAs per SM (the
-// best point of a sweep: 5.9 TB/s at 64k), exponentiated, parked in shared memory in chunks of 32
-// tiles, and summed per tile and row half in a fixed, bank-conflict-free order (bitwise
-// reproducible); the next chunk's loads are issued before the current chunk is summed.
-// The CTA then holds its block-row(s) of A' in shared memory, optionally writes them out, and
-// warp 0 ranks them (warp_select_row) and writes the CSR lists. HBM-bound:
-// 4 * 128 * ceil(L/128) * ceil(L/64) bytes read per (batch, head).
+// One CTA owns one 128-row query tile of one (batch, head), i.e. one, two or four query blocks.
+// Statistics are read with 16-byte loads (four consecutive rows of one key block; the layout
+// [bh][128-row query tile][key block][row] makes a CTA's reads one contiguous run), eight in flight
+// per thread and six CTAs per SM (the best point of a sweep: 5.9 TB/s at 64k), exponentiated,
+// parked in shared memory in chunks of 32 key blocks, and summed per key block and 32-row quarter
+// in a fixed, bank-conflict-free order (bitwise reproducible); the next chunk's loads are issued
+// before the current chunk is summed. The quarters are then combined into the CTA's block-row(s)
+// of A', which are optionally written out, and one warp per block-row ranks it (warp_select_row)
+// and writes the CSR list. HBM-bound: 4 * 128 * ceil(L/128) * (L / block_size) bytes read per
+// (batch, head).
 #include "internal.h"
 #include "topk_device.cuh"
 
@@ -33,45 +34,45 @@ constexpr int kRows = 128;
 constexpr int kInFlight = SPARSED_POOL_IN_FLIGHT;  // 16-byte loads each thread keeps in flight
 constexpr int kChunk = 4 * kInFlight;  // tiles per transposition chunk: one batch of loads per thread
 constexpr int kPitch = kRows + 4;   // floats per chunk row: keeps float4 stores aligned
-constexpr int kMaxTiles = 2048;     // seq_len <= 131072
+constexpr int kMaxBlocks = 2048;    // key blocks per row: seq_len <= 2048 * block_size
 
-// Shared memory (dynamic, sized for the actual sequence): the transposition chunk, the per-tile
-// mass of rows 0-63 / 64-127, the ordered keys of this CTA's block-row(s), the top-k histogram.
+// Shared memory (dynamic, sized for the actual sequence): the transposition chunk, the per-block
+// mass of each 32-row quarter of the query tile, the ordered keys of this CTA's block-row(s), one
+// top-k histogram per block-row.
 struct PoolSmem {
-  float* chunk;                     // [tile in chunk][kPitch]
-  float* tile_sum[2];               // [row half][tile]
-  uint32_t* keys[2];
-  int* hist;
+  float* chunk;                     // [key block in chunk][kPitch]
+  float* quarter_sum;               // [32-row quarter][key block]
+  uint32_t* keys;                   // [block-row of this CTA][key block]
+  int* hist;                        // [block-row][256]
 };
 
-__host__ __device__ inline size_t pool_smem_bytes(int n_tiles, int nb) {
-  return sizeof(float) * kChunk * kPitch + sizeof(float) * 2 * n_tiles + sizeof(uint32_t) * 2 * nb +
-         sizeof(int) * 256;
+__host__ __device__ inline size_t pool_smem_bytes(int nb, int rows_here) {
+  return sizeof(float) * kChunk * kPitch + sizeof(float) * 4 * nb + sizeof(uint32_t) * rows_here * nb +
+         sizeof(int) * 256 * rows_here;
 }
 
 __global__ void __launch_bounds__(kRows, SPARSED_POOL_CTAS_PER_SM) pool_select_kernel(const PoolParams p) {
   extern __shared__ __align__(16) uint8_t pool_smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int L = p.seq_len;
-  const int n_tiles = (L + 63) / 64;
+  const int bs = p.block_size;
+  const int nb = L / bs;                    // key blocks per row = statistics per row
+  const int rows_here = kRows / bs;         // block-rows of A' this CTA produces: 1, 2 or 4
   PoolSmem sm;
   {
     float* f = reinterpret_cast<float*>(pool_smem_raw);
     sm.chunk = f;
     f += kChunk * kPitch;
-    sm.tile_sum[0] = f;
-    sm.tile_sum[1] = f + n_tiles;
-    f += 2 * n_tiles;
-    const int nb_ = L / p.block_size;
-    sm.keys[0] = reinterpret_cast<uint32_t*>(f);
-    sm.keys[1] = sm.keys[0] + nb_;
-    sm.hist = reinterpret_cast<int*>(sm.keys[1] + nb_);
+    sm.quarter_sum = f;
+    f += 4 * nb;
+    sm.keys = reinterpret_cast<uint32_t*>(f);
+    sm.hist = reinterpret_cast<int*>(sm.keys + rows_here * nb);
   }
   const int num_q_tiles = (L + kRows - 1) / kRows;
   const int q_tile = blockIdx.x % num_q_tiles;
   const int bh = blockIdx.x / num_q_tiles;
   // Loading: lane l owns rows 4l..4l+3 of the query tile (one 16-byte load covers them), warp w
-  // takes tiles w, w+4, ... of the chunk. seq_len is a multiple of 32 here, so a group of four
+  // takes key blocks w, w+4, ... of the chunk. seq_len is a multiple of 32 here, so a group of four
   // rows is valid or invalid as a whole and 16-byte aligned.
   const int row4 = q_tile * kRows + lane * 4;
   const bool rows_valid = row4 < L;
@@ -81,16 +82,17 @@ __global__ void __launch_bounds__(kRows, SPARSED_POOL_CTAS_PER_SM) pool_select_k
     const float c = 1.44269504088896341f;
     lse2 = make_float4(t.x * c, t.y * c, t.z * c, t.w * c);
   }
-  // statistics layout [bh][query tile][key tile][128 rows]: this CTA's share is one contiguous run
-  const float* src = p.tile_lse + (static_cast<int64_t>(bh) * num_q_tiles + q_tile) * n_tiles * kRows + lane * 4;
+  // statistics layout [bh][query tile][key block][128 rows]: this CTA's share is one contiguous run
+  const float* src = p.tile_lse + (static_cast<int64_t>(bh) * num_q_tiles + q_tile) * nb * kRows + lane * 4;
 
-  // One batch = this thread's kInFlight loads of a chunk (warp w takes tiles w, w+4, ... of it). The
-  // next chunk's batch is issued before the current chunk is summed, so loads stay in flight
+  // One batch = this thread's kInFlight loads of a chunk (warp w takes key blocks w, w+4, ... of it).
+  // The next chunk's batch is issued before the current chunk is summed, so loads stay in flight
   // through the shared-memory phase.
   static_assert(kChunk == 4 * kInFlight, "one batch of loads per thread covers one chunk");
+  static_assert(kChunk == 32, "the summation assigns one key block of the chunk to each lane");
   float4 v[kInFlight];
   auto issue = [&](int c0) {
-    const int n_here = min(kChunk, n_tiles - c0);
+    const int n_here = min(kChunk, nb - c0);
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
       const int t = warp + 4 * u;
@@ -100,8 +102,8 @@ __global__ void __launch_bounds__(kRows, SPARSED_POOL_CTAS_PER_SM) pool_select_k
     }
   };
   issue(0);
-  for (int c0 = 0; c0 < n_tiles; c0 += kChunk) {
-    const int n_here = min(kChunk, n_tiles - c0);
+  for (int c0 = 0; c0 < nb; c0 += kChunk) {
+    const int n_here = min(kChunk, nb - c0);
 #pragma unroll
     for (int u = 0; u < kInFlight; ++u) {
       const int t = warp + 4 * u;
@@ -112,69 +114,72 @@ __global__ void __launch_bounds__(kRows, SPARSED_POOL_CTAS_PER_SM) pool_select_k
       }
     }
     __syncthreads();
-    if (c0 + kChunk < n_tiles) issue(c0 + kChunk);
+    if (c0 + kChunk < nb) issue(c0 + kChunk);
     {
-      // Summing: thread j < 64 adds rows 0-63 of tile j, thread j + 64 rows 64-127. Each thread
-      // starts at its own rotation of the 64 rows so that a warp's reads hit 32 different banks;
-      // the order is fixed per tile, so the result is reproducible.
-      const int half = tid >> 6;
-      for (int j = tid & 63; j < n_here; j += 64) {
-        const float* rowp = sm.chunk + j * kPitch + half * 64;
+      // Summing: warp w adds rows 32w..32w+31 (one quarter of the query tile), lane j key block j of
+      // the chunk. Each lane starts at its own rotation of the 32 rows so that a warp's reads hit 32
+      // different banks; the order is fixed per key block, so the result is reproducible.
+      const int j = lane;
+      if (j < n_here) {
+        const float* rowp = sm.chunk + j * kPitch + warp * 32;
         float acc = 0.f;
 #pragma unroll 8
-        for (int r = 0; r < 64; ++r) acc += rowp[(r + 29 * j) & 63];
-        sm.tile_sum[half][c0 + j] = acc;
+        for (int r = 0; r < 32; ++r) acc += rowp[(r + 29 * j) & 31];
+        sm.quarter_sum[warp * nb + c0 + j] = acc;
       }
     }
     __syncthreads();
   }
 
-  const int bs = p.block_size;
-  const int nb = L / bs;
   const float inv_area = 1.f / (static_cast<float>(bs) * static_cast<float>(bs));
-  const int rows_here = bs == 64 ? 2 : 1;
   for (int jb = tid; jb < nb; jb += kRows) {
+    const float q0 = sm.quarter_sum[jb], q1 = sm.quarter_sum[nb + jb], q2 = sm.quarter_sum[2 * nb + jb],
+                q3 = sm.quarter_sum[3 * nb + jb];
+    float score[4];
     if (bs == 128) {
-      const float total = (sm.tile_sum[0][2 * jb] + sm.tile_sum[1][2 * jb]) +
-                          (sm.tile_sum[0][2 * jb + 1] + sm.tile_sum[1][2 * jb + 1]);
-      const float score = total * inv_area;
-      sm.keys[0][jb] = ordered_key(score);
-      if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + q_tile) * nb + jb] = score;
+      score[0] = ((q0 + q1) + (q2 + q3)) * inv_area;
+    } else if (bs == 64) {
+      score[0] = (q0 + q1) * inv_area;
+      score[1] = (q2 + q3) * inv_area;
     } else {
+      score[0] = q0 * inv_area;
+      score[1] = q1 * inv_area;
+      score[2] = q2 * inv_area;
+      score[3] = q3 * inv_area;
+    }
 #pragma unroll
-      for (int rh = 0; rh < 2; ++rh) {
-        const int ib = q_tile * 2 + rh;
-        if (ib < nb) {
-          const float score = sm.tile_sum[rh][jb] * inv_area;
-          sm.keys[rh][jb] = ordered_key(score);
-          if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + ib) * nb + jb] = score;
-        }
+    for (int rh = 0; rh < 4; ++rh) {
+      const int ib = q_tile * rows_here + rh;
+      if (rh < rows_here && ib < nb) {
+        sm.keys[rh * nb + jb] = ordered_key(score[rh]);
+        if (p.scores != nullptr) p.scores[(static_cast<int64_t>(bh) * nb + ib) * nb + jb] = score[rh];
       }
     }
   }
   __syncthreads();
-  if (warp == 0) {
-    const int k_total = p.k_pre + p.k_gen;
-    for (int rh = 0; rh < rows_here; ++rh) {
-      const int ib = bs == 64 ? q_tile * 2 + rh : q_tile;
-      if (ib >= nb) break;
+  // one warp per block-row: isolated top-k (Eq. 5 / Eq. 6) and the CSR list
+  if (warp < rows_here) {
+    const int ib = q_tile * rows_here + warp;
+    if (ib < nb) {
+      const int k_total = p.k_pre + p.k_gen;
       const int64_t r = static_cast<int64_t>(bh) * nb + ib;
-      warp_select_row(sm.keys[rh], nb, p.pb, p.k_pre, p.k_gen, sm.hist, p.col_idx + r * k_total, lane);
+      warp_select_row(sm.keys + warp * nb, nb, p.pb, p.k_pre, p.k_gen, sm.hist + warp * 256, p.col_idx + r * k_total, lane);
       if (lane == 0) {
         p.row_ptr[r] = static_cast<int32_t>(r * k_total);
         if (r == static_cast<int64_t>(p.bh) * nb - 1) p.row_ptr[r + 1] = static_cast<int32_t>((r + 1) * k_total);
       }
-      __syncwarp();
     }
   }
 }
 
 }  // namespace
 
+int pool_select_max_blocks() { return kMaxBlocks; }
+
 cudaError_t launch_pool_select(const PoolParams& p, cudaStream_t stream) {
-  const int n_tiles = (p.seq_len + 63) / 64;
-  if (n_tiles > kMaxTiles) return cudaErrorInvalidValue;
-  const int smem = static_cast<int>(pool_smem_bytes(n_tiles, p.seq_len / p.block_size));
+  const int nb = p.seq_len / p.block_size;
+  if (nb > kMaxBlocks) return cudaErrorInvalidValue;
+  const int smem = static_cast<int>(pool_smem_bytes(nb, kRows / p.block_size));
   static SmemLimit limit;
   cudaError_t e = ensure_dynamic_smem(pool_select_kernel, smem, limit);
   if (e != cudaSuccess) return e;

@@ -104,7 +104,7 @@ def test_misaligned_side_buffers_are_refused_before_any_launch(lib):
     byref = ctypes.byref
     assert lib.sparsed_attn_full(byref(shape), ok, ok, ok, ok, off, ok, 256, None) == 3             # lse
     assert lib.sparsed_attn_full(byref(shape), ok, ok, ok, ok, None, off, 256, None) == 3            # ws
-    assert lib.sparsed_attn_full_stats(byref(shape), ok, ok, ok, ok, ok, off, ok, 256, None) == 3    # tile stats
+    assert lib.sparsed_attn_full_stats(byref(shape), 128, ok, ok, ok, ok, ok, off, ok, 256, None) == 3    # tile stats
     assert lib.sparsed_select_from_stats(byref(shape), byref(params), off, ok, byref(pat), None, ok, 256, None) == 3
     assert lib.sparsed_select_from_stats(byref(shape), byref(params), ok, off, byref(pat), None, ok, 256, None) == 3
     assert lib.sparsed_select_from_stats(byref(shape), byref(params), ok, ok, byref(pat), off, ok, 256, None) == 3

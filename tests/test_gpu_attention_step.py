@@ -1,6 +1,6 @@
 """Algorithm 1 through the single-call entry point: every step of a short denoising schedule on the GPU
-against the oracle's step-by-step composition, on inputs that change from step to step; both ways the
-switch step can select (row statistics of its own pass; the two-pass scorer for 32-token blocks)."""
+against the oracle's step-by-step composition, on inputs that change from step to step, for every block
+size (the switch step selects from the row statistics of its own full-attention pass)."""
 import numpy as np
 import pytest
 import torch
@@ -17,7 +17,7 @@ DEV = "cuda"
 @pytest.mark.parametrize("bs,L,rho,prefill,T,skip", [
     (64, 1024, 0.3, 0, 5, 0.4),        # switch at step 2, selection from the full pass's statistics
     (128, 1536, 0.25, 512, 4, 0.5),    # isolated regions, switch at step 2
-    (32, 512, 0.5, 128, 4, 0.25),      # 32-token blocks: the switch step falls back to the two-pass scorer
+    (32, 512, 0.5, 128, 4, 0.25),      # 32-token blocks: one statistic per 32 keys
     (64, 768, 0.3, 0, 3, 0.0),         # skip = 0: the first step is the switch step
 ])
 def test_schedule_through_one_entry_point(bs, L, rho, prefill, T, skip):

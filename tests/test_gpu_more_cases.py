@@ -26,8 +26,8 @@ def test_custom_scale_and_batch_two_through_all_entry_points():
     ws = sd.new_workspace(1 << 22, DEV)
     o = torch.empty_like(q)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=DEV)
-    stats = sd.new_tile_stats(q)
-    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, softmax_scale=scale)
+    stats = sd.new_tile_stats(q, 128)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, 128, softmax_scale=scale)
     o_ref, lse_ref = orc.attn_full(qd, kd, vd, scale=scale32)
     check_outputs(o, o_ref, "scaled full")
     np.testing.assert_allclose(to_f64(lse), lse_ref, atol=3e-5, rtol=3e-6)
@@ -96,8 +96,8 @@ def test_batched_long_context_settings(batch, seq_len, gen_len):
     ws = sd.new_workspace(1 << 22, DEV)
     o = torch.empty_like(q)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=DEV)
-    stats = sd.new_tile_stats(q)
-    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+    stats = sd.new_tile_stats(q, bs)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, bs)
     params = sd.make_params(bs, rho, prefill)
     kp, kg = sd.sparsed_kept_per_row(params, L)
     assert (kp, kg) == (orc.kept_per_region(pb, rho), orc.kept_per_region(nb - pb, rho))
@@ -145,8 +145,8 @@ def test_token_major_layout_through_every_entry_point():
     nb = L // bs
     ws = sd.new_workspace(1 << 22, DEV)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=DEV)
-    stats = sd.new_tile_stats(q)
-    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+    stats = sd.new_tile_stats(q, bs)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, bs)
     qd, kd, vd = to_f64(q), to_f64(k), to_f64(v)
     o_ref, lse_ref = orc.attn_full(qd, kd, vd)
     check_outputs(o, o_ref, "token-major full")

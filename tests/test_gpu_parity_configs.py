@@ -65,9 +65,9 @@ def gpu_switch_step_from_stats(q, k, v, block_size, keep_ratio, prefill_len):
     nb = L // block_size
     o = torch.empty_like(q)
     lse = torch.empty(B, Hq, L, dtype=torch.float32, device=q.device)
-    stats = sd.new_tile_stats(q)
+    stats = sd.new_tile_stats(q, block_size)
     ws = sd.new_workspace(256, q.device)
-    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws)
+    sd.sparsed_attn_full_stats(q, k, v, o, lse, stats, ws, block_size)
     params = sd.make_params(block_size, keep_ratio, prefill_len)
     kp, kg = sd.sparsed_kept_per_row(params, L)
     pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, kp + kg, q.device)
