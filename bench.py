@@ -37,19 +37,32 @@ from paper_2509_24014_b200 import synthetic as syn  # noqa: E402
 
 METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at 64k"
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/; keyed by (kernel, workload). None where no capture exists.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures of the
+# kernels, keyed by (kernel, workload): (bytes, where the figure comes from, source file of the kernel,
+# sha256 prefix of that file when the capture was taken). A figure whose kernel source has changed
+# since is reported as null with the reason, instead of going stale silently.
 NCU_DRAM_TRAFFIC = {
-    # profiles/ncu_dram_bytes_c4_step_kernels.md (1-pass capture on the full-size workload)
-    ("attn_dense_pair_kernel", "c4"): 1853606144 + 9088952832,
-    ("pool_select_kernel", "c4"): 8598426368 + 41508096,
-    ("attn_kernel<sparse>", "c4"): 1250340864 + 516116992,
-    # profiles/ncu_full_c2_all_kernels.md, profiles/ncu_full_topk_c4.md
-    ("attn_dense_pair_kernel", "c2"): 201481728 + 158934272,
-    ("pool_select_kernel", "c2"): 135332352 + 3845632,
-    ("attn_kernel<sparse>", "c2"): 156542720 + 41992192,
-    ("topk_csr_kernel", "c4"): 33585920,
 }
+
+
+def _source_digest(rel_path):
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, rel_path), "rb") as f:
+            return hashlib.sha256(f.read()).hexdigest()[:12]
+    except OSError:
+        return None
+
+
+def ncu_traffic(kernel, workload):
+    """(bytes or None, provenance string) for roofline.traffic."""
+    rec = NCU_DRAM_TRAFFIC.get((kernel, workload))
+    if rec is None:
+        return None, "no ncu capture for this kernel and workload"
+    nbytes, where, src, digest = rec
+    if _source_digest(src) != digest:
+        return None, f"stale: {src} changed since the capture ({where})"
+    return nbytes, where
 
 
 def load_peaks():
@@ -252,6 +265,104 @@ def workload_name(cfg):
 
 
 # ------------------------------------------------------------------------------ GPU arm
+def _ev():
+    return torch.cuda.Event(enable_timing=True)
+
+
+def slow_path_events(ws):
+    """Warp-level rescales of the output accumulator counted by the attention kernels in the workspace."""
+    return int(ws[32:40].view(torch.int64).item())
+
+
+def measure_config(cfg, dev, layer=0, qkv=None):
+    """Buffers and the step closure of the hot path on one workload, resident in HBM: a step is
+    attn_full_stats -> select_from_stats -> attn_sparse, optionally dropping four CUDA events.
+    cfg describes the tensors this rank holds; qkv overrides the synthetic inputs (head shards)."""
+    import paper_2509_24014_b200 as sd
+    q, k, v = qkv if qkv is not None else syn.make_qkv(cfg, dev, layer)
+    B, Hq, L, D = q.shape
+    bs, nb = cfg.block_size, cfg.num_blocks
+    o_full = torch.empty_like(q)
+    o_sparse = torch.empty_like(q)
+    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
+    params = sd.make_params(bs, cfg.keep_ratio, cfg.prefill_len)
+    k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
+    pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
+    shape_qkvo = sd.make_shape(q, k, v, o_full)
+    shape_qk = sd.make_shape(q, k)
+    ws = sd.new_workspace(256, dev)
+    tile_stats = sd.new_tile_stats(q, bs)
+
+    def step(marks=None):
+        def mark():
+            if marks is not None:
+                e = _ev(); e.record(); marks.append(e)
+        mark()
+        sd.sparsed_attn_full_stats(q, k, v, o_full, lse, tile_stats, ws, bs, shape=shape_qkvo)
+        mark()
+        sd.sparsed_select_from_stats(q, k, params, lse, tile_stats, pat, ws, shape=shape_qk)
+        mark()
+        sd.sparsed_attn_sparse(q, k, v, o_sparse, pat, ws, shape=shape_qkvo)
+        mark()
+
+    return {"q": q, "k": k, "v": v, "o_full": o_full, "o_sparse": o_sparse, "lse": lse, "params": params,
+            "kept": (k_pre, k_gen), "pat": pat, "row_ptr": row_ptr, "col_idx": col_idx, "ws": ws,
+            "tile_stats": tile_stats, "step": step, "shape_qkvo": shape_qkvo, "shape_qk": shape_qk}
+
+
+def time_config(cfg, dev, reps, warmup, peaks, layer=0):
+    """measure_config + timing, for the by-config summary. Frees the workload before returning."""
+    import paper_2509_24014_b200 as sd
+    m = measure_config(cfg, dev, layer)
+    for _ in range(warmup):
+        m["step"]()
+    torch.cuda.synchronize()
+    events = []
+    for _ in range(reps):
+        marks = []
+        m["step"](marks)
+        events.append(marks)
+    a, b = _ev(), _ev()
+    a.record()
+    for _ in range(reps):
+        sd.sparsed_attn_full(m["q"], m["k"], m["v"], m["o_full"], None, m["ws"], shape=m["shape_qkvo"])
+    b.record()
+    torch.cuda.synchronize()
+    code, where = sd.sparsed_last_device_status(m["ws"])
+    if code != 0:
+        raise RuntimeError(f"device status {code} at {where}")
+    full_stats_ms = statistics.median(e[0].elapsed_time(e[1]) for e in events)
+    select_ms = statistics.median(e[1].elapsed_time(e[2]) for e in events)
+    sparse_ms = statistics.median(e[2].elapsed_time(e[3]) for e in events)
+    dense_ms = a.elapsed_time(b) / reps
+    nnz = int(m["pat"].nnz)
+    k_pre, k_gen = m["kept"]
+    nb = cfg.num_blocks
+    peak = peaks["bf16_tflops"]
+    sparse_tf = sparse_flops(cfg, nnz) / sparse_ms / 1e9
+    dense_tf = dense_flops(cfg) / dense_ms / 1e9
+    B, Hq, L, D = m["q"].shape
+    # How often the softmax had to rescale its accumulator (logits outgrew the running maximum), per
+    # warp-level softmax group (32 query rows x 64 keys), separately for the dense and the sparse kernel.
+    sd.sparsed_workspace_init(m["ws"])
+    sd.sparsed_attn_full(m["q"], m["k"], m["v"], m["o_full"], None, m["ws"], shape=m["shape_qkvo"])
+    torch.cuda.synchronize()
+    ev_dense = slow_path_events(m["ws"])
+    sd.sparsed_attn_sparse(m["q"], m["k"], m["v"], m["o_sparse"], m["pat"], m["ws"], shape=m["shape_qkvo"])
+    torch.cuda.synchronize()
+    ev_sparse = slow_path_events(m["ws"]) - ev_dense
+    groups_dense = B * Hq * ((L + 31) // 32) * ((L + 63) // 64)
+    groups_sparse = nnz * max(1, cfg.block_size // 32) * max(1, cfg.block_size // 64)
+    out = {"workload": workload_name(cfg), "plant_norm": cfg.plant_norm, "kept_per_row": [k_pre, k_gen], "nnz": nnz,
+           "dense_ms": dense_ms, "dense_tflops": dense_tf, "dense_frac_of_burst": dense_tf / peak,
+           "dense_with_stats_ms": full_stats_ms, "select_from_stats_ms": select_ms,
+           "sparse_ms": sparse_ms, "sparse_tflops": sparse_tf, "sparse_frac_of_burst": sparse_tf / peak,
+           "speedup_vs_dense": dense_ms / sparse_ms, "ideal_speedup": nb / (k_pre + k_gen),
+           "softmax_rescale_fraction_dense": ev_dense / groups_dense,
+           "softmax_rescale_fraction_sparse": ev_sparse / groups_sparse, "reps": reps}
+    return out
+
+
 def run_ours(args, cfg):
     import paper_2509_24014_b200 as sd
 
@@ -277,43 +388,34 @@ def run_ours(args, cfg):
     sd.load_library()
     peaks = load_peaks()
 
-    cfg_r = cfg.with_(seed=replicas.replica_seed(cfg.seed, rank))
-    q, k, v = syn.make_qkv(cfg_r, dev)
+    shard_heads = args.shard == "heads" and world > 1
+    if shard_heads:
+        # one layer split over the ranks by heads (whole GQA groups): same seed everywhere, each rank
+        # keeps its own heads; total work is fixed as N grows
+        hq = replicas.shard_heads(cfg.heads_q, cfg.heads_kv, world, rank)
+        hkv = replicas.shard_kv_heads(cfg.heads_kv, world, rank)
+        qf, kf, vf = syn.make_qkv(cfg, dev)
+        qkv = (qf[:, hq.start:hq.stop].contiguous(), kf[:, hkv.start:hkv.stop].contiguous(),
+               vf[:, hkv.start:hkv.stop].contiguous())
+        del qf, kf, vf
+        torch.cuda.empty_cache()
+        cfg_local = cfg.with_(heads_q=len(hq), heads_kv=len(hkv))
+        m = measure_config(cfg_local, dev, qkv=qkv)
+        del qkv
+    else:
+        cfg_local = cfg.with_(seed=replicas.replica_seed(cfg.seed, rank))
+        m = measure_config(cfg_local, dev)
+    q, k, v, o_full, o_sparse, lse = m["q"], m["k"], m["v"], m["o_full"], m["o_sparse"], m["lse"]
     B, Hq, L, D = q.shape
     nb = cfg.num_blocks
-    o_full = torch.empty_like(q)
-    o_sparse = torch.empty_like(q)
-    lse = torch.empty(B, Hq, L, dtype=torch.float32, device=dev)
-    params = sd.make_params(cfg.block_size, cfg.keep_ratio, cfg.prefill_len)
-    k_pre, k_gen = sd.sparsed_kept_per_row(params, L)
-    pat, row_ptr, col_idx = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
-    shape_qkvo = sd.make_shape(q, k, v, o_full)
-    shape_qk = sd.make_shape(q, k)
-    ws = sd.new_workspace(sd.sparsed_workspace_bytes(sd.OP_SELECT_PATTERN, shape_qk, params), dev)
-    tile_stats = sd.new_tile_stats(q, cfg.block_size)
+    params, pat, row_ptr, col_idx, ws = m["params"], m["pat"], m["row_ptr"], m["col_idx"], m["ws"]
+    k_pre, k_gen = m["kept"]
+    shape_qkvo, shape_qk, tile_stats = m["shape_qkvo"], m["shape_qk"], m["tile_stats"]
     total_steps, skip = max(cfg.total_steps, 2), (cfg.skip if cfg.total_steps > 1 else 0.5)
     s_switch = sd.sparsed_switch_step(total_steps, skip)
-
-    def ev():
-        return torch.cuda.Event(enable_timing=True)
-
-    def step(events=None):
-        """All rows of the hot path once. Returns nothing; `events` collects 5 stream markers."""
-        marks = []
-        def mark():
-            if events is not None:
-                e = ev(); e.record(); marks.append(e)
-        mark()
-        assert sd.sparsed_schedule_mode(s_switch, total_steps, skip) == sd.MODE_FULL_AND_SELECT
-        sd.sparsed_attn_full_stats(q, k, v, o_full, lse, tile_stats, ws, cfg.block_size, shape=shape_qkvo)
-        mark()
-        sd.sparsed_select_from_stats(q, k, params, lse, tile_stats, pat, ws, shape=shape_qk)
-        mark()
-        assert sd.sparsed_schedule_mode(s_switch + 1, total_steps, skip) == sd.MODE_SPARSE
-        sd.sparsed_attn_sparse(q, k, v, o_sparse, pat, ws, shape=shape_qkvo)
-        mark()
-        if events is not None:
-            events.append(marks)
+    assert sd.sparsed_schedule_mode(s_switch, total_steps, skip) == sd.MODE_FULL_AND_SELECT
+    assert sd.sparsed_schedule_mode(s_switch + 1, total_steps, skip) == sd.MODE_SPARSE
+    step = m["step"]
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -326,10 +428,12 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     sampler.mark_begin()
     events = []
-    t_begin, t_end = ev(), ev()
+    t_begin, t_end = _ev(), _ev()
     t_begin.record()
     for _ in range(args.steps):
-        step(events)
+        marks = []
+        step(marks)
+        events.append(marks)
     t_end.record()
     torch.cuda.synchronize()
     if dist is not None:
@@ -341,34 +445,45 @@ def run_ours(args, cfg):
     if code != 0:
         raise RuntimeError(f"device status {code} at {where}")
 
-    full_ms = [m[0].elapsed_time(m[1]) for m in events]
-    select_ms = [m[1].elapsed_time(m[2]) for m in events]
-    sparse_ms = [m[2].elapsed_time(m[3]) for m in events]
+    full_ms = [e[0].elapsed_time(e[1]) for e in events]
+    select_ms = [e[1].elapsed_time(e[2]) for e in events]
+    sparse_ms = [e[2].elapsed_time(e[3]) for e in events]
     sparse_total = sum(sparse_ms)
     nnz = int(pat.nnz)
 
+    # the plain dense kernel (no statistics), the same number of calls back to back: what the
+    # sparse step's speedup is measured against
+    a, b = _ev(), _ev()
+    a.record()
+    for _ in range(args.steps):
+        sd.sparsed_attn_full(q, k, v, o_full, None, ws, shape=shape_qkvo)
+    b.record()
+    torch.cuda.synchronize()
+    dense_plain_total = a.elapsed_time(b)
+
     # max over ranks of the timed quantities
-    total_ms, sparse_total, full_total, select_total = replicas.max_over_ranks(
-        [total_ms, sparse_total, sum(full_ms), sum(select_ms)], dist, dev)
+    total_ms, sparse_total, full_total, select_total, dense_plain_total = replicas.max_over_ranks(
+        [total_ms, sparse_total, sum(full_ms), sum(select_ms), dense_plain_total], dist, dev)
 
     n = args.steps
-    value = world * n * sparse_flops(cfg, nnz) / (sparse_total * 1e-3) / 1e12
-    dense_tflops = world * n * dense_flops(cfg) / (full_total * 1e-3) / 1e12
+    cfg_work = cfg_local          # the work one rank did
+    value = world * n * sparse_flops(cfg_work, nnz) / (sparse_total * 1e-3) / 1e12
+    dense_tflops = world * n * dense_flops(cfg_work) / (dense_plain_total * 1e-3) / 1e12
+    dense_stats_tflops = world * n * dense_flops(cfg_work) / (full_total * 1e-3) / 1e12
     per_gpu_sparse = value / world
-    per_gpu_dense = dense_tflops / world
 
     # ---- end to end through the public API with host buffers (rank-local, then max) -------
     e2e_steps = max(1, min(args.steps, 3))
-    hq, hk, hv = (t.to("cpu").pin_memory() for t in (q, k, v))
+    hq_, hk_, hv_ = (t.to("cpu").pin_memory() for t in (q, k, v))
     ho = torch.empty(o_sparse.shape, dtype=o_sparse.dtype).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+    h2d = sum(t.numel() * t.element_size() for t in (hq_, hk_, hv_))
     d2h = ho.numel() * ho.element_size()
     torch.cuda.synchronize()
-    e0, e1 = ev(), ev()
+    e0, e1 = _ev(), _ev()
     from paper_2509_24014_b200.host_api import HostSparseAttention
-    host_plan = HostSparseAttention(hq, hk, row_ptr, col_idx, cfg.block_size, dev)
+    host_plan = HostSparseAttention(hq_, hk_, row_ptr, col_idx, cfg.block_size, dev)
     def e2e_once():
-        host_plan.run(hq, hk, hv, ho)
+        host_plan.run(hq_, hk_, hv_, ho)
     e2e_once()
     torch.cuda.synchronize()
     assert torch.equal(ho.to(dev), o_sparse), "host-buffer path disagrees with the resident path"
@@ -383,7 +498,7 @@ def run_ours(args, cfg):
     e2e_ms = e0.elapsed_time(e1)
     e2e_ms = replicas.max_over_ranks([e2e_ms], dist, dev)[0]
     del host_plan
-    e2e_value = world * e2e_steps * sparse_flops(cfg, nnz) / (e2e_ms * 1e-3) / 1e12
+    e2e_value = world * e2e_steps * sparse_flops(cfg_work, nnz) / (e2e_ms * 1e-3) / 1e12
 
     if rank != 0:
         if dist is not None:
@@ -396,22 +511,23 @@ def run_ours(args, cfg):
     def tensor_roofline(name, flops_per_launch, ms_list, launches_per_step=1):
         ms = sum(ms_list) / (len(ms_list) * launches_per_step)
         ach = flops_per_launch / (ms * 1e-3) / 1e12
+        traffic, source = ncu_traffic(name, cfg.name)
         return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                 "frac": ach / peak, "peak_source": f"bf16 burst, {tag}",
                 "frac_of_sustained": ach / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
-                "avg_launch_ms": ms, "traffic": NCU_DRAM_TRAFFIC.get((name, cfg.name))}
+                "avg_launch_ms": ms, "traffic": traffic, "traffic_source": source}
 
     def topk_roofline():
         """The ranking/compaction kernel alone (sparsed_select_from_scores) on this workload's A',
         HBM-bound by design; L2 is flushed before each launch by writing a 512 MB buffer."""
         scores = torch.empty(B, Hq, nb, nb, dtype=torch.float32, device=dev)
-        sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse, scores_out=scores, shape=shape_qk)
+        sd.sparsed_select_from_stats(q, k, params, lse, tile_stats, pat, ws, scores_out=scores, shape=shape_qk)
         flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
         pat2, rp2, ci2 = sd.new_pattern(B, Hq, nb, k_pre + k_gen, dev)
         times = []
         for _ in range(5):
             flush.fill_(1)
-            a, b = ev(), ev()
+            a, b = _ev(), _ev()
             a.record()
             sd.sparsed_select_from_scores(scores, params, pat2, ws)
             b.record()
@@ -421,42 +537,29 @@ def run_ours(args, cfg):
         ms = min(times[1:])
         nbytes = B * Hq * (4 * nb * nb + 4 * nb * (k_pre + k_gen) + 4 * nb)
         ach = nbytes / (ms * 1e-3) / 1e9
+        traffic, source = ncu_traffic("topk_csr_kernel", cfg.name)
         return {"kernel": "topk_csr_kernel (stand-alone, not in the step)", "bound": "hbm", "achieved": ach,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                 "peak_source": f"HBM copy, {tag}", "avg_launch_ms": ms, "algorithmic_bytes": nbytes,
-                "traffic": NCU_DRAM_TRAFFIC.get(("topk_csr_kernel", cfg.name)),
+                "traffic": traffic, "traffic_source": source,
                 "note": "event time of a single launch includes launch latency; L2 flushed before it"}
 
-    def two_pass_select():
-        """The alternative selection path (a second Q K^T pass: pooled scoring with its fused
-        top-k), timed outside the step for comparison; a dense contraction of 2*L^2*D per head."""
-        times = []
-        for _ in range(3):
-            a, b = ev(), ev()
-            a.record()
-            sd.sparsed_select_pattern(q, k, params, pat, ws, lse=lse, shape=shape_qk)
-            b.record()
-            torch.cuda.synchronize()
-            times.append(a.elapsed_time(b))
-        r = tensor_roofline("score_kernel (two-pass selection, not in the step)", dense_flops(cfg) / 2, times[1:])
-        return r
-
-    roof_dense = tensor_roofline("attn_dense_pair_kernel", dense_flops(cfg), full_ms)
-    roof_sparse = tensor_roofline("attn_kernel<sparse>", sparse_flops(cfg, nnz), sparse_ms)
-    # selection = pooled-scoring kernel (a dense QK^T contraction, 2*L^2*D per head) + top-k/CSR kernel
+    roof_dense = tensor_roofline("attn_kernel<dense>", dense_flops(cfg_work), full_ms)
+    roof_sparse = tensor_roofline("attn_kernel<sparse>", sparse_flops(cfg_work, nnz), sparse_ms)
     launches_per_step = 3
-    # selection from the recorded statistics is HBM-bound: it reads 4*L*ceil(L/64) bytes per head
+    # selection from the recorded statistics is HBM-bound: it reads 4 * L * L / block_size bytes per head
     stats_bytes = tile_stats.numel() * 4 + lse.numel() * 4 + 4 * nnz + 4 * (B * Hq * nb + 1)
     sel_ms = sum(select_ms) / len(select_ms)
     sel_gbs = stats_bytes / (sel_ms * 1e-3) / 1e9
+    traffic, source = ncu_traffic("pool_select_kernel", cfg.name)
     roof_select = {"kernel": "pool_select_kernel", "bound": "hbm", "achieved": sel_gbs, "peak": peaks["hbm_gbs"],
                    "unit": "GB/s", "frac": sel_gbs / peaks["hbm_gbs"], "peak_source": f"HBM copy, {tag}",
                    "avg_launch_ms": sel_ms, "algorithmic_bytes": stats_bytes,
-                   "traffic": NCU_DRAM_TRAFFIC.get(("pool_select_kernel", cfg.name))}
-    roof_topk = topk_roofline()
-    roof_two_pass = two_pass_select()
+                   "algorithmic_bytes_of_selection_alone": B * Hq * (4 * nb * nb + 4 * nb * (k_pre + k_gen) + 4 * nb),
+                   "traffic": traffic, "traffic_source": source}
+    roof_topk = topk_roofline() if not shard_heads else None
     dominant = max((roof_dense, roof_select, roof_sparse), key=lambda r: r["avg_launch_ms"])
-    roof_all = [roof_dense, roof_select, roof_sparse, roof_two_pass, roof_topk]
+    roof_all = [r for r in (roof_dense, roof_select, roof_sparse, roof_topk) if r is not None]
 
     # ---- CPU oracle beside it (bounded sample of the same workload) ----------------------
     cpu = None
@@ -464,7 +567,7 @@ def run_ours(args, cfg):
         rp_h = row_ptr.cpu().numpy()
         ci_h = col_idx.cpu().numpy()
         n_rows = args.cpu_rows
-        val, secs, rows, threads = oracle_sparse_sample(cfg, hq, hk, hv, rp_h, ci_h, n_rows)
+        val, secs, rows, threads = oracle_sparse_sample(cfg_work, hq_, hk_, hv_, rp_h, ci_h, n_rows)
         cpu = {"value": val, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
                "sample": f"oracle masked attention (fp64 numpy) on {rows} seeded (head, query block) rows of "
                          f"{Hq * nb}, GPU-selected pattern, {secs:.1f} s; kept-block FLOPs / time",
@@ -472,41 +575,71 @@ def run_ours(args, cfg):
                "cpu_seconds_extrapolated": secs * (B * Hq * nb) / rows,
                "gpu_ms": {"attn_full_stats": full_total / n, "select_from_stats": select_total / n,
                           "attn_sparse": sparse_total / n},
-               "other_stages": oracle_stage_samples(cfg, hq, hk, hv, max(4, n_rows // 8))}
+               "other_stages": oracle_stage_samples(cfg_work, hq_, hk_, hv_, max(4, n_rows // 8))}
 
     qkvo_gb = 4 * q.numel() * 2 / 1e9
     loop = None
+    by_config = None
+    extra = {}
+    del hq_, hk_, hv_, ho, tile_stats, o_full, o_sparse, q, k, v, m, step
+    torch.cuda.empty_cache()
     if world == 1 and not args.no_schedule_loop and cfg.total_steps > 1:
         # the workload's real schedule (sustained sparse phase, pattern reuse), same process
-        del hq, hk, hv, ho, tile_stats, o_full, o_sparse, q, k, v
-        torch.cuda.empty_cache()
         loop = run_schedule_loop(args, cfg, emit=False)
+        torch.cuda.empty_cache()
+    if world == 1 and not args.no_by_config and cfg.name == "c4":
+        # the other workloads, a sharp-logit arm of this one and the paper's short-context setting
+        by_config = {}
+        for name in ("c2", "c3"):
+            by_config[name] = time_config(syn.CONFIGS[name], dev, 20, 3, peaks)
+            torch.cuda.empty_cache()
+        c5 = syn.CONFIGS["c5"]
+        by_config["c5"] = time_config(c5, dev, 10, 3, peaks)
+        torch.cuda.empty_cache()
+        by_config["c5"]["schedule_loop"] = run_schedule_loop(args, c5, emit=False)
+        torch.cuda.empty_cache()
+        extra["sharp_logits"] = time_config(cfg.with_(plant_norm=12.0), dev, 5, 2, peaks)
+        extra["sharp_logits"]["what"] = ("the headline workload with the planted vectors at norm 12 (logit boost 12.7): "
+                                         "sink, stripe and band heads with logit ranges of 10+, where the softmax's "
+                                         "rescaling path fires; softmax_rescale_fraction = warp-level rescales per "
+                                         "(32 rows x 64 keys) softmax group")
+        torch.cuda.empty_cache()
+        short = syn.AttnConfig("short32", 8, 32, 32, 4096, 128, 32, 0.5, 2048, seed=32)
+        extra["short_context_block32"] = time_config(short, dev, 20, 3, peaks)
+        extra["short_context_block32"]["what"] = ("the paper's short-context setting: block 32, keep 50 %, L = 4096 "
+                                                  "(2048 prompt + 2048 generation), batch 8 x 32 heads; TFLOP/s "
+                                                  "counted on kept-block FLOPs only")
+        torch.cuda.empty_cache()
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": n, "warmup": args.warmup,
-        "ms_per_step": total_ms / n, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": total_ms / n, "higher_is_better": True, "scaling": "strong" if shard_heads else "weak",
+        "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "step": "attn_full_stats -> select_from_stats -> attn_sparse",
                    "kept_per_row": [k_pre, k_gen], "nnz": nnz, "density": nnz / (B * Hq * nb * nb),
                    "l2": "inputs larger than L2 (Q,K,V,O = %.2f GB per pass)" % qkvo_gb,
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": ("heads sharded over ranks, no collective" if shard_heads else
+                                   "replicas only" if world > 1 else "single GPU")},
         "pct_bf16_peak": 100.0 * per_gpu_sparse / peak,
         "pct_bf16_peak_sustained": 100.0 * per_gpu_sparse / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
         "pct_bf16_nominal_2250": 100.0 * per_gpu_sparse / 2250.0,
-        "dense_tflops": dense_tflops,
-        "speedup_vs_dense": full_total / sparse_total, "ideal_speedup": nb / (k_pre + k_gen),
+        "dense_tflops": dense_tflops, "dense_with_stats_tflops": dense_stats_tflops,
+        "speedup_vs_dense": dense_plain_total / sparse_total,
+        "speedup_vs_dense_with_stats": full_total / sparse_total, "ideal_speedup": nb / (k_pre + k_gen),
         "phase_ms": {"attn_full_stats": full_total / n, "select_from_stats": select_total / n,
-                     "attn_sparse": sparse_total / n},
+                     "attn_sparse": sparse_total / n, "attn_full_plain (timed after the steps)": dense_plain_total / n},
         "roofline": dominant, "roofline_by_kernel": roof_all,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "pinned host Q,K,V -> device, sparsed_attn_sparse, O -> pinned host; chunks of 4 kv heads on 3 streams", "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": launches_per_step * n,
-        "launches_per_step": {"attn_dense_pair_kernel (+ tile statistics)": 1,
+        "launches_per_step": {"attn_kernel<dense> (+ row statistics)": 1,
                               "pool_select_kernel (pooling + top-k + CSR)": 1, "attn_kernel<sparse>": 1},
-        "clocks": clocks, "peaks": peaks, "schedule_loop": loop,
+        "clocks": clocks, "peaks": peaks, "schedule_loop": loop, "by_config": by_config,
     }
+    line.update(extra)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -540,10 +673,6 @@ def run_topk_only(args, cfg):
     print(json.dumps({"kernel": "topk_csr_kernel", "workload": workload_name(cfg), "rows": B * Hq * nb, "nb": nb,
                       "ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms / 1e6,
                       "frac_of_hbm_peak": nbytes / ms / 1e6 / peaks["hbm_gbs"], "l2": "flushed before each launch"}))
-
-
-def _ev():
-    return torch.cuda.Event(enable_timing=True)
 
 
 def run_schedule_loop(args, cfg, emit=True):
@@ -831,6 +960,10 @@ def main():
                     help="run the config's whole denoising schedule (c4: 64 steps, c5: 4 layers x 256 steps)")
     ap.add_argument("--all-full", action="store_true", help="with --schedule-loop: also time all-full attention")
     ap.add_argument("--no-schedule-loop", action="store_true", help="skip the schedule-loop summary of the default run")
+    ap.add_argument("--no-by-config", action="store_true",
+                    help="skip the summary of the other workloads (c2, c3, c5, sharp logits, block 32)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="with --gpus N > 1: independent replicas (default) or one layer's heads split over the ranks")
     ap.add_argument("--sweep", action="store_true", help="keep-ratio / isolation / ablation / comparison-pattern timings")
     ap.add_argument("--estimate-recall", action="store_true",
                     help="exact selection vs the block-mean estimate: time, recall, kept mass, output error")

@@ -1,6 +1,6 @@
-// Block-sparse attention (Eq. 3 / Eq. 4 times V; the "Sparse Reusing" branch of Algorithm 1) for
-// head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a. (Dense attention has its own
-// two-tiles-per-CTA kernel in attention_dense.cu.)
+// Attention for head_dim 128, bf16 in / bf16 out, fp32 softmax, on sm_100a, from one kernel:
+// dense bidirectional attention (Eq. 1 times V; the full-attention branch of Algorithm 1) and
+// block-sparse attention over CSR block lists (Eq. 3 / Eq. 4 times V; the "Sparse Reusing" branch).
 //
 // One CTA owns 128 consecutive query rows of one (batch, head) and streams 64-key tiles through a
 // warp-specialised pipeline:
@@ -21,6 +21,9 @@
 // Two CTAs fit on one SM (at most 112 KB of shared memory and 256 tensor-memory columns each).
 //
 // Where the keys come from:
+//   * dense: every 64-key tile of the sequence in order; the last one may be ragged (any seq_len).
+//     Optional outputs: the rows' LSE, and the per-row statistics of each group of 32 / 64 / 128 keys
+//     from which the switch step's pooled scores are formed.
 //   * 128-key blocks: the 128 query rows are one query block; its CSR list is walked as it is,
 //     two tiles per block.
 //   * 64- and 32-key blocks: the 128 query rows are two / four consecutive query blocks with lists
@@ -44,10 +47,6 @@ constexpr int kTmemCols = 256;
 constexpr int kColS = 0;      // two S buffers of 64 fp32 columns; P (bf16 pairs) reuses the first 32
 constexpr int kColO = 128;    // O accumulator (fp32, 128 columns)
 constexpr int kMaxPackedBlocks = 2048;   // key blocks per row the union walk can hold (64- and 32-key blocks)
-#ifndef SPARSED_ATTN_POLY_EVERY
-#define SPARSED_ATTN_POLY_EVERY 0
-#endif
-constexpr int kPolyEvery = SPARSED_ATTN_POLY_EVERY;  // every n-th exponential on the FMA pipes (0 = none)
 
 // Debug builds (-DSPARSED_TIMELINE) record clock64 stamps of one CTA's pipeline roles after the
 // workspace status block: 3 regions of 2048 int64 (softmax thread 0, UMMA thread, TMA thread).
@@ -78,10 +77,12 @@ struct AttnSmem {
   uint16_t union_ids[kPacked ? kMaxPackedBlocks : 2];      // packed: the union, ascending
 };
 
-template <int kBlock>
+// kDense: walk every key tile of the sequence (kBlock must be 128 then; no block lists are read).
+template <int kBlock, bool kDense>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+  static_assert(!kDense || kBlock == 128, "the dense walk uses the unpacked layout");
   using Smem = AttnSmem<kBlock>;
   constexpr bool kPacked = Smem::kPacked;
   constexpr int kSlots = Smem::kSlots;
@@ -109,12 +110,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const int kv_head = head / p.group;
   const int q_row0 = q_tile * kTileM;
   const int qb0 = q_tile * kGroups;                          // first query block of this CTA
-  const int groups_here = min(kGroups, p.num_blocks - qb0);  // the last CTA of a head may hold fewer
-  const int r0 = bh * p.num_blocks + qb0;                    // CSR row of query block qb0
+  const int groups_here = kDense ? 1 : min(kGroups, p.num_blocks - qb0);  // the last CTA of a head may hold fewer
+  const int r0 = bh * p.num_blocks + qb0;                                 // CSR row of query block qb0
 
-  // list_begin / list_len: the CSR entries of this CTA's query blocks (adjacent rows are adjacent in col_idx)
-  const int list_begin = __ldg(p.row_ptr + r0);
-  const int list_len = __ldg(p.row_ptr + r0 + groups_here) - list_begin;
+  // list_begin / list_len: the CSR entries of this CTA's query blocks (adjacent rows are adjacent in
+  // col_idx); the dense walk has ceil(seq_len / 64) tiles instead
+  int list_begin = 0, list_len = (p.seq_len + kTileN - 1) / kTileN;
+  if constexpr (!kDense) {
+    list_begin = __ldg(p.row_ptr + r0);
+    list_len = __ldg(p.row_ptr + r0 + groups_here) - list_begin;
+  }
 
   // ---- set-up --------------------------------------------------------------------------
   // The producer warp starts the load nothing else depends on before the CTA-wide set-up has
@@ -207,9 +212,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   const uint32_t tO = tmem + kColO;
-  const int n_entries = kPacked ? sm.n_union : list_len;   // key blocks this CTA walks
-  const int num_tiles =
-      kBlocksPerTile == 1 ? n_entries * kTilesPerBlock : (n_entries + kBlocksPerTile - 1) / kBlocksPerTile;
+  const int n_entries = kPacked ? sm.n_union : list_len;   // key blocks this CTA walks (dense: key tiles)
+  const int num_tiles = kDense ? list_len
+                        : kBlocksPerTile == 1 ? n_entries * kTilesPerBlock
+                                              : (n_entries + kBlocksPerTile - 1) / kBlocksPerTile;
 
   // Warps 4 and 5 run their loops with all 32 lanes converged and let one elected lane issue
   // the TMA / UMMA instructions: their operands then stay on the uniform datapath.
@@ -220,14 +226,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       bool ok = true;
       // unpacked walk: block ids are fetched 32 at a time, one per lane
       int list_ids = 0;
-      if constexpr (!kPacked) {
+      if constexpr (!kPacked && !kDense) {
         if (lane < n_entries) list_ids = __ldg(p.col_idx + list_begin + lane);
       }
       for (int t = 0; ok && t < num_tiles; ++t) {
         // entry of this tile's (first) block in the walked list
         const int e = kBlocksPerTile == 1 ? t / kTilesPerBlock : kBlocksPerTile * t;
         int kv_row0, kv_row1 = 0, blocks_here = 1;
-        if constexpr (!kPacked) {
+        if constexpr (kDense) {
+          kv_row0 = t * kTileN;
+        } else if constexpr (!kPacked) {
           if (e > 0 && (e & 31) == 0 && t % kTilesPerBlock == 0)
             list_ids = (e + lane < n_entries) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
           kv_row0 = __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock + (t % kTilesPerBlock) * kTileN;
@@ -323,6 +331,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     bool ok = true;
     TL_DECL(0)
     RowState st{-INFINITY, 0.f};
+    RowStatWriter stats;
+    if constexpr (kDense) {
+      const int groups = (p.seq_len + p.stat_keys - 1) / p.stat_keys;
+      float* first = nullptr;
+      if (p.tile_lse != nullptr && q_row0 + tid < p.seq_len)
+        first = p.tile_lse + (static_cast<int64_t>(bh) * p.num_q_tiles + q_tile) * groups * kTileM + tid;
+      stats.init(first, p.stat_keys, groups);
+    }
     for (int t = 0; t < num_tiles; ++t) {
       TL(1);
       // S_t is ready when the Q K^T batch that read ring slot 2t has completed
@@ -350,6 +366,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       }
       uint32_t pk[32];
+      float2 stat_sums = make_float2(0.f, 0.f);
       if (kPacked && !keep0 && !keep1) {
         // nothing of this tile is kept by this warp's query block: P = 0, no exponentials
 #pragma unroll
@@ -360,6 +377,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tmem_ld32(tS + 32, r1);
         tmem_wait_ld();
         TL(3);
+        if constexpr (kDense) {
+          const int valid_cols = p.seq_len - t * kTileN;   // ragged tail of the sequence
+          if (valid_cols < kTileN) mask_columns_from(r0, r1, valid_cols);
+        }
         if constexpr (kPacked) {
           if (!keep0) {
 #pragma unroll
@@ -373,7 +394,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         float2 sums;
         bool exact = (st.m == -INFINITY);   // nothing accumulated yet: no reference maximum to try
         if (!__all_sync(0xffffffffu, exact)) {
-          sums = softmax_group_fast<kPolyEvery>(r0, r1, scale_log2, st.m, pk);
+          sums = softmax_group_fast(r0, r1, scale_log2, st.m, pk);
           exact = !(sums.x + sums.y <= 256.0f);   // logits outgrew the running maximum (or NaN)
         }
         if (__any_sync(0xffffffffu, exact)) {
@@ -391,6 +412,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
         }
         st.l += sums.x + sums.y;
+        stat_sums = sums;
       }
       TL(4);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
@@ -398,6 +420,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tc_fence_before();
       mbar_arrive(&sm.p_full[t & 1]);
       TL(5);
+      // the statistic is worked out after P has been handed over: off the S -> P -> P V chain
+      if constexpr (kDense) stats.put(t, stat_sums, st.m);
     }
 
     // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
@@ -412,6 +436,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + batch * p.o_stride_b + head * p.o_stride_h +
                            static_cast<int64_t>(row) * p.o_stride_t;
     store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
+    if constexpr (kDense) {
+      if (p.lse != nullptr && row_valid)
+        p.lse[static_cast<int64_t>(bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
+    }
   }
 
   // ---- teardown ------------------------------------------------------------------------
@@ -423,10 +451,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int kBlock>
+template <int kBlock, bool kDense>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kBlock>;
+  auto kernel = attn_kernel<kBlock, kDense>;
   const int smem = static_cast<int>(sizeof(AttnSmem<kBlock>));
   static SmemLimit limit;  // per template instantiation
   cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
@@ -445,9 +473,15 @@ int attn_sparse_max_blocks(int block_size) { return block_size < kTileM ? kMaxPa
 // p.num_q_tiles = ceil(seq_len / 128), p.num_blocks = seq_len / block_size.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<64>(tq, tk, tv, p, batch, stream);
-  return launch<32>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<128, false>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<64, false>(tq, tk, tv, p, batch, stream);
+  return launch<32, false>(tq, tk, tv, p, batch, stream);
+}
+
+// Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
+cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                              const AttnParams& p, int batch, cudaStream_t stream) {
+  return launch<128, true>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed

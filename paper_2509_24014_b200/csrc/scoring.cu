@@ -24,15 +24,11 @@ constexpr int kTile = 128;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;
 constexpr int kStages = 2;
-#ifndef SPARSED_SCORE_POLY_EVERY
-#define SPARSED_SCORE_POLY_EVERY 0
-#endif
-constexpr int kScorePolyEvery = SPARSED_SCORE_POLY_EVERY;  // every n-th exponential on the FMA pipes (0 = none)
 
 struct ScoreSmem {
   alignas(1024) __nv_bfloat16 q[2][kTile * 64];
   alignas(1024) __nv_bfloat16 k[kStages][2][kTile * 64];
-  uint64_t q_full, k_full[kStages], k_empty[kStages], s_full[2], s_empty[2], partial_full[4];
+  uint64_t q_full, k_full[kStages], s_full[2], s_empty[2], partial_full[4];
   float partial[4][4][2];  // [tile % 4][warp][column half]
   uint32_t keys[2][kFusedTopkMaxBlocks];  // ordered keys of the block-row(s) of this CTA (fused top-k)
   int hist[256];
@@ -63,10 +59,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 
   if (tid == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.k_full[s], 1);
-      mbar_init(&sm.k_empty[s], 1);
-    }
+    static_assert(kStages == 2, "K stage and S buffer of a tile share one index and one completion barrier");
+    for (int s = 0; s < kStages; ++s) mbar_init(&sm.k_full[s], 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.s_full[s], 1);
       mbar_init(&sm.s_empty[s], 128);
@@ -94,7 +88,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
       for (int it = 0; it < num_tiles; ++it) {
         const int s = it % kStages;
         const int use = it / kStages;
-        if (use > 0 && !mbar_wait(&sm.k_empty[s], (use - 1) & 1, &sm.abort_flag, p.status, 40)) break;
+        // the stage's previous K tile has been read once the S buffer of the same index is complete
+        if (use > 0 && !mbar_wait(&sm.s_full[s], (use - 1) & 1, &sm.abort_flag, p.status, 40)) break;
         mbar_expect_tx(&sm.k_full[s], kTile * kHeadDim * 2);
         tma_load_4d(sm.k[s][0], &tm_k, &sm.k_full[s], 0, it * kTile, kv_head, batch);
         tma_load_4d(sm.k[s][1], &tm_k, &sm.k_full[s], 64, it * kTile, kv_head, batch);
@@ -118,8 +113,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           umma_ss(tmem + buf * kTile, umma_smem_desc_sw128(q_addr[kk >> 2] + off, 16, 1024),
                   umma_smem_desc_sw128(k_addr[kk >> 2] + off, 16, 1024), idesc, kk > 0);
         }
-        umma_commit(&sm.k_empty[s]);
-        umma_commit(&sm.s_full[buf]);
+        umma_commit(&sm.s_full[buf]);   // one commit: "S ready" for the softmax warps, "K stage free" for the producer
       }
     }
   } else {
@@ -186,7 +180,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
           float acc = 0.f;
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            acc += tile_exp2<kScorePolyEvery>(fmaf(__uint_as_float(r[j]), scale_log2, -lse2), j);
+            acc += fast_exp2(fmaf(__uint_as_float(r[j]), scale_log2, -lse2));
           half_sum[c >> 1] += acc;
           quarter[c] = acc;
         }
