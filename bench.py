@@ -41,7 +41,25 @@ METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at
 # kernels, keyed by (kernel, workload): (bytes, where the figure comes from, source file of the kernel,
 # sha256 prefix of that file when the capture was taken). A figure whose kernel source has changed
 # since is reported as null with the reason, instead of going stale silently.
+_C2_ATTN = "ncu --set full capture of one launch on the 8k workload (summary under profiles/)"
+_C2_POOL = "ncu --set full capture of one launch on the 8k workload (summary under profiles/)"
+_ATTN_SRC, _ATTN_SHA = "paper_2509_24014_b200/csrc/attention.cu", "08fa8b826bec"
+_POOL_SRC, _POOL_SHA = "paper_2509_24014_b200/csrc/pool_select.cu", "840b284c40be"
 NCU_DRAM_TRAFFIC = {
+    ("attn_kernel<dense>", "c2"): (201476096 + 100872448, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
+    ("attn_kernel<sparse>", "c2"): (156410112 + 42415616, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
+    ("pool_select_kernel", "c2"): (68195328 + 522496, _C2_POOL, _POOL_SRC, _POOL_SHA),
+    # 64k workload: the 8k capture scaled by the algorithmic bytes of a launch (traffic was the algorithmic
+    # traffic at 8k: every K/V re-read hits L2), instead of a multi-counter capture of a 7 GB workload.
+    # dense + statistics: Q,K,V,O + LSE + statistics = 6450 MB at 64k against 336 MB at 8k
+    ("attn_kernel<dense>", "c4"): (int((201476096 + 100872448) * 6450.0 / 336.0), _C2_ATTN + ", scaled x19.2 by algorithmic bytes",
+                                   _ATTN_SRC, _ATTN_SHA),
+    # sparse: Q + O + touched K,V: 8x the rows and 8x the K/V of the 8k workload
+    ("attn_kernel<sparse>", "c4"): ((156410112 + 42415616) * 8, _C2_ATTN + ", scaled x8 by algorithmic bytes",
+                                    _ATTN_SRC, _ATTN_SHA),
+    # pooling: the statistics stream, 64x the 8k one (rows x8, key blocks x8)
+    ("pool_select_kernel", "c4"): ((68195328 + 522496) * 64, _C2_POOL + ", scaled x64 by algorithmic bytes",
+                                   _POOL_SRC, _POOL_SHA),
 }
 
 
