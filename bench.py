@@ -871,7 +871,7 @@ def run_sweep(args, cfg):
     sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws)
     sp_ms = timed(lambda: sd.sparsed_attn_sparse(q, k, v, o, pat, ws))
     resel_ms = timed(lambda: sd.sparsed_select_pattern(q, k, params, pat, ws, lse=None), reps=3)
-    T, skip = max(cfg.total_steps, 2), cfg.skip if cfg.total_steps > 1 else 0.2
+    T, skip = (cfg.total_steps, cfg.skip) if cfg.total_steps > 1 else (64, 0.2)   # workloads without a schedule: the 64k one's
     s_sw = sd.sparsed_switch_step(T, skip)
     sel_ms = timed(lambda: sd.sparsed_select_from_stats(q, k, params, lse, stats, pat, ws))
     total_sparsed = (s_sw - 1) * full_ms + full_stats_ms + sel_ms + (T - s_sw) * sp_ms
