@@ -277,8 +277,10 @@ sparsed_status sparsed_build_window_pattern(int32_t batch, int32_t heads_q, int3
 sparsed_status sparsed_pattern_validate(const sparsed_pattern *pattern, void *ws, size_t ws_bytes,
                                         void *cuda_stream);
 
-/* Reads the device status word (synchronises the stream). code 0 = fine, 1 = a wait ran out;
- * `where` identifies the wait. Returns SPARSED_ERR_DEVICE_TIMEOUT if code != 0. */
+/* Reads the device status word (synchronises the stream). code 0 = fine, 1 = a bounded wait ran out
+ * (`where` identifies the wait), 2 = a kernel found its shared memory misaligned, 3 = sparsed_attn_sparse
+ * met a row_ptr entry that points outside col_idx (that query block's rows were written as zeros).
+ * Returns SPARSED_ERR_DEVICE_TIMEOUT if code != 0. */
 sparsed_status sparsed_last_device_status(void *ws, void *cuda_stream, int32_t *code, int32_t *where);
 
 /*

@@ -370,6 +370,7 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   p.scale_log2 = rs.scale_log2;
   p.row_ptr = nullptr;
   p.col_idx = nullptr;
+  p.col_capacity = 0;
   p.status = static_cast<DeviceStatus*>(ws);
   cudaError_t e = launch_attn_dense(tq, tk, tv, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
@@ -522,6 +523,7 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   p.scale_log2 = rs.scale_log2;
   p.row_ptr = pattern->row_ptr;
   p.col_idx = pattern->col_idx;
+  p.col_capacity = pattern->col_capacity;
   p.status = static_cast<DeviceStatus*>(ws);
   cudaError_t e = launch_attn_sparse(tq, tk, tv, p, shape->batch, bs, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);

@@ -119,14 +119,52 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if constexpr (!kDense) {
     list_begin = __ldg(p.row_ptr + r0);
     list_len = __ldg(p.row_ptr + r0 + groups_here) - list_begin;
+    if (list_begin < 0 || list_len < 0 || static_cast<int64_t>(list_begin) + list_len > p.col_capacity) {
+      // row_ptr points outside col_idx: not followed; the rows get zeros and the status word says why
+      if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, 3) == 0) p.status->where = 2;
+      list_begin = 0;
+      list_len = 0;
+    }
   }
 
   // ---- set-up --------------------------------------------------------------------------
-  // The producer warp starts the load nothing else depends on before the CTA-wide set-up has
-  // finished: the Q tile, through a barrier it initialises itself.
+  // The producer warp owns the barriers of its own loads, so it can start them before the CTA-wide
+  // set-up (tensor-memory allocation, the other barriers) has finished: the Q tile, the first block
+  // ids of the list and, when the list needs no preparation, the first ring-full of K/V tiles. The
+  // chain row_ptr -> col_idx -> first K tile -> first MMA is what a short list's run time consists of.
+  int list_ids = 0;     // unpacked walk: lane i holds the block id of list entry 32 * chunk + i
+  int loads_issued = 0; // K/V loads already issued by the producer (load 2t is K_t, load 2t+1 is V_t)
+  // rows [kv_row0, +64) (or two 32-row blocks at kv_row0 / kv_row1) of K (which = 0) or V into `slot`
+  auto issue_load = [&](int slot, int which, int kv_row0, int kv_row1, int blocks_here) {
+    if (elect_one_sync()) {
+      const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+      if constexpr (kBlocksPerTile == 1) {
+        mbar_expect_tx(&sm.kv_full[slot], kTileN * kHeadDim * 2);
+        tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
+        tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+      } else {
+        // tensor-map boxes are 32 rows here; block b of the tile lands at rows 32 b
+        mbar_expect_tx(&sm.kv_full[slot], blocks_here * kBlock * kHeadDim * 2);
+        tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
+        tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+        if (blocks_here == 2) {
+          tma_load_4d(sm.kv[slot][0] + kBlock * 64, tm, &sm.kv_full[slot], 0, kv_row1, kv_head, batch);
+          tma_load_4d(sm.kv[slot][1] + kBlock * 64, tm, &sm.kv_full[slot], 64, kv_row1, kv_head, batch);
+        }
+      }
+    }
+    __syncwarp();
+  };
+  // first key row of tile t in the unpacked walks
+  auto unpacked_row = [&](int t) -> int {
+    if constexpr (kDense) return t * kTileN;
+    const int e = t / kTilesPerBlock;
+    return __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock + (t % kTilesPerBlock) * kTileN;
+  };
   if (warp == 4) {
     if (lane == 0) {
       mbar_init(&sm.q_full, 1);
+      for (int s = 0; s < kSlots; ++s) mbar_init(&sm.kv_full[s], 1);
       mbar_fence_init();
     }
     __syncwarp();
@@ -140,13 +178,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
       }
       __syncwarp();
+      if constexpr (!kPacked) {
+        if constexpr (!kDense) {
+          if (lane < list_len) list_ids = __ldg(p.col_idx + list_begin + lane);
+        }
+        const int tiles = kDense ? list_len : list_len * kTilesPerBlock;
+        const int first = min(2 * tiles, kSlots);   // entry 0..15 of the list at most: within the first chunk
+        for (; loads_issued < first; ++loads_issued)
+          issue_load(loads_issued, loads_issued & 1, unpacked_row(loads_issued >> 1), 0, 1);
+      }
     }
   }
   if (tid == 0) {
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(&sm.kv_full[s], 1);
-      mbar_init(&sm.done[s], 1);
-    }
+    for (int s = 0; s < kSlots; ++s) mbar_init(&sm.done[s], 1);
     for (int s = 0; s < 2; ++s) mbar_init(&sm.p_full[s], kSoftmaxThreads);
     sm.abort_flag = 0;
     sm.n_union = 0;
@@ -224,22 +268,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     if (num_tiles > 0) {
       TL_DECL(2)
       bool ok = true;
-      // unpacked walk: block ids are fetched 32 at a time, one per lane
-      int list_ids = 0;
-      if constexpr (!kPacked && !kDense) {
-        if (lane < n_entries) list_ids = __ldg(p.col_idx + list_begin + lane);
-      }
-      for (int t = 0; ok && t < num_tiles; ++t) {
-        // entry of this tile's (first) block in the walked list
-        const int e = kBlocksPerTile == 1 ? t / kTilesPerBlock : kBlocksPerTile * t;
+      // load i: K (even) or V (odd) of tile i / 2; a slot is reused every kSlots loads
+      for (int i = loads_issued; ok && i < 2 * num_tiles; ++i) {
+        const int t = i >> 1;
         int kv_row0, kv_row1 = 0, blocks_here = 1;
-        if constexpr (kDense) {
-          kv_row0 = t * kTileN;
-        } else if constexpr (!kPacked) {
-          if (e > 0 && (e & 31) == 0 && t % kTilesPerBlock == 0)
-            list_ids = (e + lane < n_entries) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
-          kv_row0 = __shfl_sync(0xffffffffu, list_ids, e & 31) * kBlock + (t % kTilesPerBlock) * kTileN;
+        if constexpr (!kPacked) {
+          if constexpr (!kDense) {
+            // block ids are fetched 32 at a time, one per lane, when the walk enters a new chunk
+            const int e = t / kTilesPerBlock;
+            if ((i & 1) == 0 && e > 0 && (e & 31) == 0 && t % kTilesPerBlock == 0)
+              list_ids = (e + lane < n_entries) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
+          }
+          kv_row0 = unpacked_row(t);
         } else {
+          const int e = kBlocksPerTile * t;
           kv_row0 = static_cast<int>(sm.union_ids[e]) * kBlock;
           if (kBlocksPerTile > 1 && e + 1 < n_entries) {
             // two 32-key blocks side by side in one 64-key tile; an odd union leaves the last tile half filled
@@ -247,36 +289,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             blocks_here = 2;
           }
         }
-        // load 2t (K_t) and load 2t+1 (V_t); a slot is reused every kSlots loads
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {
-          const int i = 2 * t + which;
-          const int slot = i % kSlots;
-          TL(20 + which);
-          if (i >= kSlots) {
-            ok = mbar_wait(&sm.done[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-          }
-          if (elect_one_sync()) {
-            const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
-            if constexpr (kBlocksPerTile == 1) {
-              mbar_expect_tx(&sm.kv_full[slot], kTileN * kHeadDim * 2);
-              tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
-              tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
-            } else {
-              // tensor-map boxes are 32 rows here; block b of the tile lands at rows 32 b
-              mbar_expect_tx(&sm.kv_full[slot], blocks_here * kBlock * kHeadDim * 2);
-              tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
-              tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
-              if (blocks_here == 2) {
-                tma_load_4d(sm.kv[slot][0] + kBlock * 64, tm, &sm.kv_full[slot], 0, kv_row1, kv_head, batch);
-                tma_load_4d(sm.kv[slot][1] + kBlock * 64, tm, &sm.kv_full[slot], 64, kv_row1, kv_head, batch);
-              }
-            }
-          }
-          __syncwarp();
+        const int slot = i % kSlots;
+        TL(20 + (i & 1));
+        if (i >= kSlots) {
+          ok = mbar_wait(&sm.done[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
         }
+        issue_load(slot, i & 1, kv_row0, kv_row1, blocks_here);
         TL(22);
       }
     }

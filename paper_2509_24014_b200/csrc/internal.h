@@ -50,6 +50,7 @@ struct AttnParams {
   float scale_log2;        // softmax scale * log2(e)
   const int32_t* row_ptr;  // sparse only
   const int32_t* col_idx;  // sparse only
+  int64_t col_capacity;    // sparse only: entries of col_idx that may be read
   DeviceStatus* status;
 };
 

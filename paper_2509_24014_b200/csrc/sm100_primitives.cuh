@@ -15,7 +15,8 @@
 namespace sparsed {
 
 // ----------------------------------------------------------------------------
-// Device status word: {code, where}.  code 0 = fine, 1 = a wait ran out.
+// Device status word: {code, where}.  code 0 = fine, 1 = a wait ran out, 2 = misaligned shared
+// memory, 3 = a CSR row pointer outside the column array.
 // ----------------------------------------------------------------------------
 struct DeviceStatus {
   int code;

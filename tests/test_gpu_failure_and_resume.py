@@ -42,3 +42,35 @@ def test_resume_sparse_phase_from_saved_pattern(tmp_path):
     assert torch.equal(rp2, row_ptr) and torch.equal(ci2, col_idx[: pat.nnz]) and pat2.num_blocks == pat.num_blocks
     assert sd.sparsed_pattern_validate(pat2, sd.new_workspace(256, DEV))
     assert torch.equal(gpu_sparse(q, k, v, pat2), o1)
+
+
+@pytest.mark.parametrize("bs", [128, 32])
+def test_row_pointers_outside_the_column_array_are_not_followed(bs):
+    """A corrupt row_ptr (pointing past col_idx, or backwards) must not make the sparse kernel read out
+    of bounds: the affected query blocks come back as zeros, the status word reads code 3, every other
+    query block is computed as usual, and the context stays usable."""
+    cfg = syn.AttnConfig("g", 1, 2, 2, 1024, 128, bs, 0.3, 0, seed=93)
+    q, k, v = syn.make_qkv(cfg, DEV)
+    pat, row_ptr, col_idx, _ = gpu_select(q, k, bs, 0.3, 0)
+    good = gpu_sparse(q, k, v, pat)
+    nb = 1024 // bs
+    group = 128 // bs                                   # query blocks that share a 128-row tile
+    bad_rp = row_ptr.clone()
+    victim = 3 * group                                  # first query block of the fourth query tile of head 0
+    bad_rp[victim + group] = 10 ** 9                    # its tile's list would end a billion entries in
+    bad = sd.pattern_from_csr(bad_rp, col_idx, bs, nb, 1, 2)
+    o = torch.full_like(q, float("nan"))
+    ws = sd.new_workspace(256, DEV)
+    sd.sparsed_attn_sparse(q, k, v, o, bad, ws)
+    torch.cuda.synchronize()
+    code, where = sd.sparsed_last_device_status(ws)
+    assert (code, where) == (3, 2)
+    rows = slice(victim * bs, (victim + group) * bs)
+    assert torch.all(o[0, 0, rows] == 0)
+    keep = torch.ones(1024, dtype=torch.bool, device=DEV)
+    keep[rows] = False
+    nxt = slice((victim + group) * bs, (victim + 2 * group) * bs)   # the next tile starts at the corrupt entry too
+    keep[nxt] = False
+    assert torch.equal(o[0, 0, keep], good[0, 0, keep]) and torch.equal(o[0, 1], good[0, 1])
+    sd.sparsed_workspace_init(ws)
+    assert torch.equal(gpu_sparse(q, k, v, pat), good)
