@@ -137,6 +137,20 @@ sparsed_status check_arch() {
   return major == 10 ? SPARSED_OK : SPARSED_ERR_ARCH;
 }
 
+// CTAs of the attention kernel that are resident on the current device at once (two per SM), cached per
+// device; 0 if the SM count cannot be read (the kernel then gets one CTA per query tile).
+int attn_max_ctas() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  static std::atomic<int> cached[64];
+  int n = (dev >= 0 && dev < 64) ? cached[dev].load(std::memory_order_relaxed) : 0;
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64) cached[dev].store(n, std::memory_order_relaxed);
+  }
+  return 2 * n;
+}
+
 sparsed_status check_shape(const sparsed_shape* s, bool need_v_o, Resolved* r) {
   if (s == nullptr) return SPARSED_ERR_INVALID_ARG;
   if (s->batch < 1 || s->heads_q < 1 || s->heads_kv < 1 || s->seq_len < 1) return SPARSED_ERR_INVALID_ARG;
@@ -367,6 +381,8 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   p.group = shape->heads_q / shape->heads_kv;
   p.num_q_tiles = (shape->seq_len + 127) / 128;
   p.num_blocks = 0;
+  p.num_items = shape->batch * shape->heads_q * p.num_q_tiles;
+  p.max_ctas = 0;   // dense: one CTA per query tile (running on into further tiles measured 1-2 % slower here)
   p.scale_log2 = rs.scale_log2;
   p.row_ptr = nullptr;
   p.col_idx = nullptr;
@@ -520,6 +536,10 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   p.group = shape->heads_q / shape->heads_kv;
   p.num_q_tiles = (shape->seq_len + 127) / 128;
   p.num_blocks = pattern->num_blocks;
+  p.num_items = shape->batch * shape->heads_q * p.num_q_tiles;
+  // block lists: as many CTAs as are resident at once, each running through its share of the query tiles, so
+  // that only a CTA's first tile pays the start-up chain (+16 % at 4 blocks per row, +5 % at 14, +1 % at 52)
+  p.max_ctas = attn_max_ctas();
   p.scale_log2 = rs.scale_log2;
   p.row_ptr = pattern->row_ptr;
   p.col_idx = pattern->col_idx;

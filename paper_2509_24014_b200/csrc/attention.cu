@@ -101,57 +101,85 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const int warp = tid >> 5;
   const int lane = tid & 31;
 
-  // ---- work item -----------------------------------------------------------------------
-  // num_q_tiles = 128-row query tiles per (batch, head); num_blocks = pattern blocks per row
-  const int q_tile = blockIdx.x % p.num_q_tiles;
-  const int bh = blockIdx.x / p.num_q_tiles;
-  const int head = bh % p.heads_q;
-  const int batch = bh / p.heads_q;
-  const int kv_head = head / p.group;
-  const int q_row0 = q_tile * kTileM;
-  const int qb0 = q_tile * kGroups;                          // first query block of this CTA
-  const int groups_here = kDense ? 1 : min(kGroups, p.num_blocks - qb0);  // the last CTA of a head may hold fewer
-  const int r0 = bh * p.num_blocks + qb0;                                 // CSR row of query block qb0
-
-  // list_begin / list_len: the CSR entries of this CTA's query blocks (adjacent rows are adjacent in
-  // col_idx); the dense walk has ceil(seq_len / 64) tiles instead
-  int list_begin = 0, list_len = (p.seq_len + kTileN - 1) / kTileN;
-  if constexpr (!kDense) {
-    list_begin = __ldg(p.row_ptr + r0);
-    list_len = __ldg(p.row_ptr + r0 + groups_here) - list_begin;
-    if (list_begin < 0 || list_len < 0 || static_cast<int64_t>(list_begin) + list_len > p.col_capacity) {
-      // row_ptr points outside col_idx: not followed; the rows get zeros and the status word says why
-      if (threadIdx.x == 0 && atomicCAS(&p.status->code, 0, 3) == 0) p.status->where = 2;
-      list_begin = 0;
-      list_len = 0;
+  // ---- work items ----------------------------------------------------------------------
+  // An item is one 128-row query tile of one (batch, head). A CTA takes items blockIdx.x,
+  // blockIdx.x + gridDim.x, ... ; the host launches either one CTA per item or (dense and 128-key
+  // blocks only) as many CTAs as fit on the device at once, in which case each role of the pipeline
+  // runs on into its next item on its own: the producer loads the next Q, list and K/V tiles while
+  // the softmax warps are still in the previous item's last tiles and epilogue, so the start-up
+  // chain row_ptr -> col_idx -> first K tile -> first MMA of all but a CTA's first item is hidden.
+  // Every counter below (loads, tiles, Q loads) runs on across items and all roles compute the same
+  // values, so ring slots, S buffers and barrier phases simply continue.
+  struct Item {
+    int q_tile, bh, head, batch, kv_head, q_row0, groups_here, r0;
+    int list_begin, list_len;   // CSR entries of the item's query blocks; dense: key tiles of the sequence
+  };
+  const int n_items = p.num_items;
+  auto describe = [&](int item) -> Item {
+    Item it;
+    it.q_tile = item % p.num_q_tiles;
+    it.bh = item / p.num_q_tiles;
+    it.head = it.bh % p.heads_q;
+    it.batch = it.bh / p.heads_q;
+    it.kv_head = it.head / p.group;
+    it.q_row0 = it.q_tile * kTileM;
+    const int qb0 = it.q_tile * kGroups;                                   // first query block of the item
+    it.groups_here = kDense ? 1 : min(kGroups, p.num_blocks - qb0);        // the last tile of a head may hold fewer
+    it.r0 = it.bh * p.num_blocks + qb0;                                    // CSR row of query block qb0
+    it.list_begin = 0;
+    it.list_len = (p.seq_len + kTileN - 1) / kTileN;
+    if constexpr (!kDense) {
+      // adjacent rows are adjacent in col_idx, so the item's lists are one run of entries
+      it.list_begin = __ldg(p.row_ptr + it.r0);
+      it.list_len = __ldg(p.row_ptr + it.r0 + it.groups_here) - it.list_begin;
+      if (it.list_begin < 0 || it.list_len < 0 ||
+          static_cast<int64_t>(it.list_begin) + it.list_len > p.col_capacity) {
+        // row_ptr points outside col_idx: not followed; the rows get zeros and the status word says why
+        if (atomicCAS(&p.status->code, 0, 3) == 0) p.status->where = 2;
+        it.list_begin = 0;
+        it.list_len = 0;
+      }
     }
-  }
+    return it;
+  };
+  // tiles of an item in the unpacked walks (the packed walk counts its union instead)
+  auto unpacked_tiles = [&](const Item& it) -> int { return kDense ? it.list_len : it.list_len * kTilesPerBlock; };
+
+  const int first_item = blockIdx.x;
+  Item cur = describe(first_item);
 
   // ---- set-up --------------------------------------------------------------------------
   // The producer warp owns the barriers of its own loads, so it can start them before the CTA-wide
   // set-up (tensor-memory allocation, the other barriers) has finished: the Q tile, the first block
-  // ids of the list and, when the list needs no preparation, the first ring-full of K/V tiles. The
-  // chain row_ptr -> col_idx -> first K tile -> first MMA is what a short list's run time consists of.
+  // ids of the list and, when the list needs no preparation, the first ring-full of K/V tiles.
   int list_ids = 0;     // unpacked walk: lane i holds the block id of list entry 32 * chunk + i
-  int loads_issued = 0; // K/V loads already issued by the producer (load 2t is K_t, load 2t+1 is V_t)
+  int loads_issued = 0; // K/V loads of the first item already issued by the producer before the set-up barrier
   // rows [kv_row0, +64) (or two 32-row blocks at kv_row0 / kv_row1) of K (which = 0) or V into `slot`
-  auto issue_load = [&](int slot, int which, int kv_row0, int kv_row1, int blocks_here) {
+  auto issue_load = [&](const Item& it, int slot, int which, int kv_row0, int kv_row1, int blocks_here) {
     if (elect_one_sync()) {
       const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
       if constexpr (kBlocksPerTile == 1) {
         mbar_expect_tx(&sm.kv_full[slot], kTileN * kHeadDim * 2);
-        tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
-        tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+        tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, it.kv_head, it.batch);
+        tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, it.kv_head, it.batch);
       } else {
         // tensor-map boxes are 32 rows here; block b of the tile lands at rows 32 b
         mbar_expect_tx(&sm.kv_full[slot], blocks_here * kBlock * kHeadDim * 2);
-        tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, kv_head, batch);
-        tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, kv_head, batch);
+        tma_load_4d(sm.kv[slot][0], tm, &sm.kv_full[slot], 0, kv_row0, it.kv_head, it.batch);
+        tma_load_4d(sm.kv[slot][1], tm, &sm.kv_full[slot], 64, kv_row0, it.kv_head, it.batch);
         if (blocks_here == 2) {
-          tma_load_4d(sm.kv[slot][0] + kBlock * 64, tm, &sm.kv_full[slot], 0, kv_row1, kv_head, batch);
-          tma_load_4d(sm.kv[slot][1] + kBlock * 64, tm, &sm.kv_full[slot], 64, kv_row1, kv_head, batch);
+          tma_load_4d(sm.kv[slot][0] + kBlock * 64, tm, &sm.kv_full[slot], 0, kv_row1, it.kv_head, it.batch);
+          tma_load_4d(sm.kv[slot][1] + kBlock * 64, tm, &sm.kv_full[slot], 64, kv_row1, it.kv_head, it.batch);
         }
       }
+    }
+    __syncwarp();
+  };
+  auto issue_q_load = [&](const Item& it) {
+    if (elect_one_sync()) {
+      mbar_expect_tx(&sm.q_full, kTileM * kHeadDim * 2);   // rows beyond the sequence arrive as zeros
+      tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, it.q_row0, it.head, it.batch);
+      tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, it.q_row0, it.head, it.batch);
     }
     __syncwarp();
   };
@@ -168,24 +196,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       mbar_fence_init();
     }
     __syncwarp();
-    if (list_len > 0) {
-      if (elect_one_sync()) {
-        tma_prefetch_desc(&tm_q);
-        tma_prefetch_desc(&tm_k);
-        tma_prefetch_desc(&tm_v);
-        mbar_expect_tx(&sm.q_full, kTileM * kHeadDim * 2);   // rows beyond the sequence arrive as zeros
-        tma_load_4d(sm.q[0], &tm_q, &sm.q_full, 0, q_row0, head, batch);
-        tma_load_4d(sm.q[1], &tm_q, &sm.q_full, 64, q_row0, head, batch);
-      }
-      __syncwarp();
+    if (elect_one_sync()) {
+      tma_prefetch_desc(&tm_q);
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_v);
+    }
+    __syncwarp();
+    if (cur.list_len > 0) {
+      issue_q_load(cur);
       if constexpr (!kPacked) {
         if constexpr (!kDense) {
-          if (lane < list_len) list_ids = __ldg(p.col_idx + list_begin + lane);
+          if (lane < cur.list_len) list_ids = __ldg(p.col_idx + cur.list_begin + lane);
         }
-        const int tiles = kDense ? list_len : list_len * kTilesPerBlock;
-        const int first = min(2 * tiles, kSlots);   // entry 0..15 of the list at most: within the first chunk
+        const int first = min(2 * unpacked_tiles(cur), kSlots);   // list entries 0..2 at most: within the first chunk
         for (; loads_issued < first; ++loads_issued)
-          issue_load(loads_issued, loads_issued & 1, unpacked_row(loads_issued >> 1), 0, 1);
+          issue_load(cur, loads_issued, loads_issued & 1, unpacked_row(loads_issued >> 1), 0, 1);
       }
     }
   }
@@ -209,14 +234,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     tmem_relinquish();
   }
   if constexpr (kPacked) {
-    // One bitmap per query block, then their union as an ascending list.
+    // (one item per CTA here) One bitmap per query block, then their union as an ascending list.
     const int words = (p.num_blocks + 31) >> 5;
     for (int i = tid; i < kGroups * Smem::kWords; i += kThreads) (&sm.member[0][0])[i] = 0u;
     __syncthreads();
     int bound[kGroups];   // bound[g] = first CSR entry after query block g's list
 #pragma unroll
-    for (int g = 0; g < kGroups; ++g) bound[g] = __ldg(p.row_ptr + r0 + min(g + 1, groups_here));
-    for (int e = list_begin + tid; e < list_begin + list_len; e += kThreads) {
+    for (int g = 0; g < kGroups; ++g) bound[g] = __ldg(p.row_ptr + cur.r0 + min(g + 1, cur.groups_here));
+    for (int e = cur.list_begin + tid; e < cur.list_begin + cur.list_len; e += kThreads) {
       const int id = __ldg(p.col_idx + e);
       int g = 0;
 #pragma unroll
@@ -256,20 +281,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
   const uint32_t tO = tmem + kColO;
-  const int n_entries = kPacked ? sm.n_union : list_len;   // key blocks this CTA walks (dense: key tiles)
-  const int num_tiles = kDense ? list_len
-                        : kBlocksPerTile == 1 ? n_entries * kTilesPerBlock
-                                              : (n_entries + kBlocksPerTile - 1) / kBlocksPerTile;
+  // key blocks an item walks (dense: key tiles) and its tiles
+  auto entries_of = [&](const Item& it) -> int { return kPacked ? sm.n_union : it.list_len; };
+  auto tiles_of = [&](const Item& it) -> int {
+    const int n = entries_of(it);
+    return kDense ? n : kBlocksPerTile == 1 ? n * kTilesPerBlock : (n + kBlocksPerTile - 1) / kBlocksPerTile;
+  };
 
   // Warps 4 and 5 run their loops with all 32 lanes converged and let one elected lane issue
   // the TMA / UMMA instructions: their operands then stay on the uniform datapath.
   if (warp == 4) {
     // =============================== TMA producer =======================================
-    if (num_tiles > 0) {
-      TL_DECL(2)
-      bool ok = true;
+    TL_DECL(2)
+    bool ok = true;
+    int load0 = 0;       // K/V loads issued for earlier items
+    int prev_tiles = 0;  // tiles of the latest earlier item that had any
+    for (int item = first_item; ok && item < n_items; item += gridDim.x) {
+      if (item != first_item) {
+        cur = describe(item);
+        if (cur.list_len > 0) {
+          if (prev_tiles > 0) {
+            // the Q buffer is free once the previous item's last Q K^T batch (which read load load0 - 2) is done
+            const int g = load0 - 2;
+            ok = mbar_wait(&sm.done[g % kSlots], (g / kSlots) & 1, &sm.abort_flag, p.status, 11);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          issue_q_load(cur);
+          if constexpr (!kPacked && !kDense) {
+            list_ids = (lane < cur.list_len) ? __ldg(p.col_idx + cur.list_begin + lane) : 0;
+          }
+        }
+      }
+      const int n_entries = entries_of(cur);
+      const int num_tiles = tiles_of(cur);
       // load i: K (even) or V (odd) of tile i / 2; a slot is reused every kSlots loads
-      for (int i = loads_issued; ok && i < 2 * num_tiles; ++i) {
+      for (int i = (item == first_item ? loads_issued : 0); ok && i < 2 * num_tiles; ++i) {
         const int t = i >> 1;
         int kv_row0, kv_row1 = 0, blocks_here = 1;
         if constexpr (!kPacked) {
@@ -277,7 +324,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             // block ids are fetched 32 at a time, one per lane, when the walk enters a new chunk
             const int e = t / kTilesPerBlock;
             if ((i & 1) == 0 && e > 0 && (e & 31) == 0 && t % kTilesPerBlock == 0)
-              list_ids = (e + lane < n_entries) ? __ldg(p.col_idx + list_begin + e + lane) : 0;
+              list_ids = (e + lane < n_entries) ? __ldg(p.col_idx + cur.list_begin + e + lane) : 0;
           }
           kv_row0 = unpacked_row(t);
         } else {
@@ -289,57 +336,74 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             blocks_here = 2;
           }
         }
-        const int slot = i % kSlots;
+        const int g = load0 + i;
+        const int slot = g % kSlots;
         TL(20 + (i & 1));
-        if (i >= kSlots) {
-          ok = mbar_wait(&sm.done[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
+        if (g >= kSlots) {
+          ok = mbar_wait(&sm.done[slot], ((g / kSlots) - 1) & 1, &sm.abort_flag, p.status, 10);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
         }
-        issue_load(slot, i & 1, kv_row0, kv_row1, blocks_here);
+        issue_load(cur, slot, i & 1, kv_row0, kv_row1, blocks_here);
         TL(22);
       }
+      load0 += 2 * num_tiles;
+      if (num_tiles > 0) prev_tiles = num_tiles;
     }
   } else if (warp == 5) {
     // =============================== UMMA issuer ========================================
-    if (num_tiles > 0) {
-      // descriptor low words: Q is fixed; K/V slots differ only in their base address
-      const uint32_t q_lo0 = umma_desc_lo(smem_u32(sm.q[0]), 16);
-      const uint32_t kv_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), 16);            // as K (K-major)
-      const uint32_t v_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), kTileN * 128);   // as V (MN-major)
-      constexpr uint32_t slot_step = (2 * kTileN * 64 * 2) >> 4;                  // 16 KB per ring slot
-      TL_DECL(1)
-      // S_t = Q K_t^T into S buffer t & 1
+    // descriptor low words: Q is fixed; K/V slots differ only in their base address
+    const uint32_t q_lo0 = umma_desc_lo(smem_u32(sm.q[0]), 16);
+    const uint32_t kv_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), 16);            // as K (K-major)
+    const uint32_t v_lo0 = umma_desc_lo(smem_u32(sm.kv[0][0]), kTileN * 128);   // as V (MN-major)
+    constexpr uint32_t slot_step = (2 * kTileN * 64 * 2) >> 4;                  // 16 KB per ring slot
+    TL_DECL(1)
+    bool ok = true;
+    int load0 = 0, tile0 = 0, q_loads = 0;   // loads / tiles / Q tiles of earlier items
+    for (int item = first_item; ok && item < n_items; item += gridDim.x) {
+      if (item != first_item) cur = describe(item);
+      const int num_tiles = tiles_of(cur);
+      if (num_tiles == 0) continue;
+      // S_t = Q K_t^T into S buffer (tile0 + t) & 1
       auto issue_qk = [&](int t) -> bool {
-        const int i = 2 * t;
-        const int slot = i % kSlots;
+        const int g = load0 + 2 * t;
+        const int slot = g % kSlots;
         TL(10);
-        bool got = mbar_wait(&sm.kv_full[slot], (i / kSlots) & 1, &sm.abort_flag, p.status, 21);
+        bool got = mbar_wait(&sm.kv_full[slot], (g / kSlots) & 1, &sm.abort_flag, p.status, 21);
         got = __all_sync(0xffffffffu, got);
         if (!got) return false;
         TL(11);
-        issue_qk64(tmem + kColS + (t & 1) * kTileN, q_lo0, kv_lo0 + slot * slot_step, &sm.done[slot]);
+        issue_qk64(tmem + kColS + ((tile0 + t) & 1) * kTileN, q_lo0, kv_lo0 + slot * slot_step, &sm.done[slot]);
         TL(12);
         return true;
       };
-      bool ok = mbar_wait(&sm.q_full, 0, &sm.abort_flag, p.status, 20);
+      ok = mbar_wait(&sm.q_full, q_loads & 1, &sm.abort_flag, p.status, 20);
       ok = __all_sync(0xffffffffu, ok);
+      ++q_loads;
       ok = ok && issue_qk(0);
       for (int t = 0; ok && t < num_tiles; ++t) {
-        // The S buffer of tile t+1 last held P_{t-1}, whose P V was issued one iteration ago,
-        // and tcgen05 operations of one thread execute in issue order.
-        if (t + 1 < num_tiles && !issue_qk(t + 1)) break;
-        const int i = 2 * t + 1;
-        const int slot = i % kSlots;
+        // The S buffer of tile t+1 last held P of the tile two before it, whose P V was issued
+        // earlier by this thread, and tcgen05 operations of one thread execute in issue order.
+        if (t + 1 < num_tiles && !issue_qk(t + 1)) {
+          ok = false;
+          break;
+        }
+        const int g = load0 + 2 * t + 1;
+        const int slot = g % kSlots;
+        const int gt = tile0 + t;
         TL(13);
-        ok = mbar_wait2(&sm.p_full[t & 1], (t >> 1) & 1, &sm.kv_full[slot], (i / kSlots) & 1, &sm.abort_flag,
+        ok = mbar_wait2(&sm.p_full[gt & 1], (gt >> 1) & 1, &sm.kv_full[slot], (g / kSlots) & 1, &sm.abort_flag,
                         p.status, 22);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         TL(14);
-        issue_pv64(tO, tmem + kColS + (t & 1) * kTileN, v_lo0 + slot * slot_step, t > 0, &sm.done[slot]);
+        // the first P V of an item overwrites O: the softmax warps handed P over after they had read the
+        // previous item's O out in their epilogue
+        issue_pv64(tO, tmem + kColS + (gt & 1) * kTileN, v_lo0 + slot * slot_step, t > 0, &sm.done[slot]);
         TL(15);
       }
+      load0 += 2 * num_tiles;
+      tile0 += num_tiles;
     }
   } else {
     // =============================== softmax / epilogue =================================
@@ -347,118 +411,130 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const float scale_log2 = p.scale_log2;
     // packed walk: this warp's 32 rows belong to one query block
     const int my_group = kPacked ? (warp * 32) / kBlock : 0;
-    const bool group_valid = my_group < groups_here;
     bool ok = true;
     TL_DECL(0)
-    RowState st{-INFINITY, 0.f};
-    RowStatWriter stats;
-    if constexpr (kDense) {
-      const int groups = (p.seq_len + p.stat_keys - 1) / p.stat_keys;
-      float* first = nullptr;
-      if (p.tile_lse != nullptr && q_row0 + tid < p.seq_len)
-        first = p.tile_lse + (static_cast<int64_t>(bh) * p.num_q_tiles + q_tile) * groups * kTileM + tid;
-      stats.init(first, p.stat_keys, groups);
-    }
-    for (int t = 0; t < num_tiles; ++t) {
-      TL(1);
-      // S_t is ready when the Q K^T batch that read ring slot 2t has completed
-      if (!mbar_wait(&sm.done[(2 * t) % kSlots], ((2 * t) / kSlots) & 1, &sm.abort_flag, p.status, 30)) {
-        ok = false;
-        break;
+    int load0 = 0, tile0 = 0;   // loads / tiles of earlier items
+    for (int item = first_item; ok && item < n_items; item += gridDim.x) {
+      if (item != first_item) cur = describe(item);
+      const int n_entries = entries_of(cur);
+      const int num_tiles = tiles_of(cur);
+      const bool group_valid = my_group < cur.groups_here;
+      RowState st{-INFINITY, 0.f};
+      RowStatWriter stats;
+      if constexpr (kDense) {
+        const int groups = (p.seq_len + p.stat_keys - 1) / p.stat_keys;
+        float* first = nullptr;
+        if (p.tile_lse != nullptr && cur.q_row0 + tid < p.seq_len)
+          first = p.tile_lse + (static_cast<int64_t>(cur.bh) * p.num_q_tiles + cur.q_tile) * groups * kTileM + tid;
+        stats.init(first, p.stat_keys, groups);
       }
-      TL(2);
-      tc_fence_after();
-      const uint32_t tS = tmem + kColS + (t & 1) * kTileN + lane_base;
-      // packed walk: which 32-column chunks of this tile hold key blocks this warp's query block kept
-      bool keep0 = true, keep1 = true;
-      if constexpr (kPacked) {
-        const int e = kBlocksPerTile * t;
-        const int id0 = sm.union_ids[e];
-        keep0 = group_valid && ((sm.member[my_group][id0 >> 5] >> (id0 & 31)) & 1u) != 0u;
-        if constexpr (kBlocksPerTile == 1) {
-          keep1 = keep0;
-        } else {
-          keep1 = false;
-          if (e + 1 < n_entries) {
-            const int id1 = sm.union_ids[e + 1];
-            keep1 = group_valid && ((sm.member[my_group][id1 >> 5] >> (id1 & 31)) & 1u) != 0u;
-          }
+      for (int t = 0; t < num_tiles; ++t) {
+        TL(1);
+        // S_t is ready when the Q K^T batch that read ring load 2t of this item has completed
+        const int gk = load0 + 2 * t;
+        if (!mbar_wait(&sm.done[gk % kSlots], (gk / kSlots) & 1, &sm.abort_flag, p.status, 30)) {
+          ok = false;
+          break;
         }
-      }
-      uint32_t pk[32];
-      float2 stat_sums = make_float2(0.f, 0.f);
-      if (kPacked && !keep0 && !keep1) {
-        // nothing of this tile is kept by this warp's query block: P = 0, no exponentials
-#pragma unroll
-        for (int j = 0; j < 32; ++j) pk[j] = 0u;
-      } else {
-        uint32_t r0[32], r1[32];
-        tmem_ld32(tS, r0);
-        tmem_ld32(tS + 32, r1);
-        tmem_wait_ld();
-        TL(3);
-        if constexpr (kDense) {
-          const int valid_cols = p.seq_len - t * kTileN;   // ragged tail of the sequence
-          if (valid_cols < kTileN) mask_columns_from(r0, r1, valid_cols);
-        }
+        TL(2);
+        tc_fence_after();
+        const int gt = tile0 + t;
+        const uint32_t tS = tmem + kColS + (gt & 1) * kTileN + lane_base;
+        // packed walk: which 32-column chunks of this tile hold key blocks this warp's query block kept
+        bool keep0 = true, keep1 = true;
         if constexpr (kPacked) {
-          if (!keep0) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r0[j] = 0xff800000u;   // -inf
-          }
-          if (!keep1) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r1[j] = 0xff800000u;
-          }
-        }
-        float2 sums;
-        bool exact = (st.m == -INFINITY);   // nothing accumulated yet: no reference maximum to try
-        if (!__all_sync(0xffffffffu, exact)) {
-          sums = softmax_group_fast(r0, r1, scale_log2, st.m, pk);
-          exact = !(sums.x + sums.y <= 256.0f);   // logits outgrew the running maximum (or NaN)
-        }
-        if (__any_sync(0xffffffffu, exact)) {
-          const float alpha = softmax_group_exact(r0, r1, scale_log2, st, pk, sums);
-          if (t > 0) {
-            // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring slot 2t-1) has drained
-            const int ip = 2 * (t - 1) + 1;
-            if (!mbar_wait(&sm.done[ip % kSlots], (ip / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
-              ok = false;
-              break;
+          const int e = kBlocksPerTile * t;
+          const int id0 = sm.union_ids[e];
+          keep0 = group_valid && ((sm.member[my_group][id0 >> 5] >> (id0 & 31)) & 1u) != 0u;
+          if constexpr (kBlocksPerTile == 1) {
+            keep1 = keep0;
+          } else {
+            keep1 = false;
+            if (e + 1 < n_entries) {
+              const int id1 = sm.union_ids[e + 1];
+              keep1 = group_valid && ((sm.member[my_group][id1 >> 5] >> (id1 & 31)) & 1u) != 0u;
             }
-            tc_fence_after();
-            rescale_accumulator_row(tO + lane_base, alpha);
-            if (p.slow_path_events != nullptr && lane == 0) atomicAdd(p.slow_path_events, 1ull);
           }
         }
-        st.l += sums.x + sums.y;
-        stat_sums = sums;
+        uint32_t pk[32];
+        float2 stat_sums = make_float2(0.f, 0.f);
+        if (kPacked && !keep0 && !keep1) {
+          // nothing of this tile is kept by this warp's query block: P = 0, no exponentials
+#pragma unroll
+          for (int j = 0; j < 32; ++j) pk[j] = 0u;
+        } else {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(tS, r0);
+          tmem_ld32(tS + 32, r1);
+          tmem_wait_ld();
+          TL(3);
+          if constexpr (kDense) {
+            const int valid_cols = p.seq_len - t * kTileN;   // ragged tail of the sequence
+            if (valid_cols < kTileN) mask_columns_from(r0, r1, valid_cols);
+          }
+          if constexpr (kPacked) {
+            if (!keep0) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r0[j] = 0xff800000u;   // -inf
+            }
+            if (!keep1) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r1[j] = 0xff800000u;
+            }
+          }
+          float2 sums;
+          bool exact = (st.m == -INFINITY);   // nothing accumulated yet: no reference maximum to try
+          if (!__all_sync(0xffffffffu, exact)) {
+            sums = softmax_group_fast(r0, r1, scale_log2, st.m, pk);
+            exact = !(sums.x + sums.y <= 256.0f);   // logits outgrew the running maximum (or NaN)
+          }
+          if (__any_sync(0xffffffffu, exact)) {
+            const float alpha = softmax_group_exact(r0, r1, scale_log2, st, pk, sums);
+            if (t > 0) {
+              // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring load 2t-1) has drained
+              const int gp = load0 + 2 * (t - 1) + 1;
+              if (!mbar_wait(&sm.done[gp % kSlots], (gp / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
+                ok = false;
+                break;
+              }
+              tc_fence_after();
+              rescale_accumulator_row(tO + lane_base, alpha);
+              if (p.slow_path_events != nullptr && lane == 0) atomicAdd(p.slow_path_events, 1ull);
+            }
+          }
+          st.l += sums.x + sums.y;
+          stat_sums = sums;
+        }
+        TL(4);
+        tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&sm.p_full[gt & 1]);
+        TL(5);
+        // the statistic is worked out after P has been handed over: off the S -> P -> P V chain
+        if constexpr (kDense) stats.put(t, stat_sums, st.m);
       }
-      TL(4);
-      tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&sm.p_full[t & 1]);
-      TL(5);
-      // the statistic is worked out after P has been handed over: off the S -> P -> P V chain
-      if constexpr (kDense) stats.put(t, stat_sums, st.m);
-    }
+      if (!ok) break;
 
-    // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
-    if (ok && num_tiles > 0) {
-      const int il = 2 * (num_tiles - 1) + 1;   // the last P V read ring slot il
-      ok = mbar_wait(&sm.done[il % kSlots], (il / kSlots) & 1, &sm.abort_flag, p.status, 31);
-    }
-    tc_fence_after();
-    const int row = q_row0 + tid;
-    const bool row_valid = row < p.seq_len;
-    const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
-    __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + batch * p.o_stride_b + head * p.o_stride_h +
-                           static_cast<int64_t>(row) * p.o_stride_t;
-    store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
-    if constexpr (kDense) {
-      if (p.lse != nullptr && row_valid)
-        p.lse[static_cast<int64_t>(bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
+      // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
+      if (num_tiles > 0) {
+        const int gl = load0 + 2 * (num_tiles - 1) + 1;   // the last P V read this load's slot
+        ok = mbar_wait(&sm.done[gl % kSlots], (gl / kSlots) & 1, &sm.abort_flag, p.status, 31);
+      }
+      tc_fence_after();
+      const int row = cur.q_row0 + tid;
+      const bool row_valid = row < p.seq_len;
+      const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
+      __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + cur.batch * p.o_stride_b +
+                             cur.head * p.o_stride_h + static_cast<int64_t>(row) * p.o_stride_t;
+      store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
+      if constexpr (kDense) {
+        if (p.lse != nullptr && row_valid)
+          p.lse[static_cast<int64_t>(cur.bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
+      }
+      tc_fence_before();   // the next item's first P V overwrites O: order these reads before its hand-over
+      load0 += 2 * num_tiles;
+      tile0 += num_tiles;
     }
   }
 
@@ -479,8 +555,11 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
   static SmemLimit limit;  // per template instantiation
   cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
   if (e != cudaSuccess) return e;
-  const long long ctas = static_cast<long long>(batch) * p.heads_q * p.num_q_tiles;
+  // one CTA per item, or (p.max_ctas > 0; not for the packed walk, which prepares its union once per CTA)
+  // at most that many CTAs, each running through its share of the items
+  long long ctas = p.num_items;
   if (ctas <= 0) return cudaSuccess;
+  if (kBlock == kTileM && p.max_ctas > 0 && ctas > p.max_ctas) ctas = p.max_ctas;
   kernel<<<static_cast<unsigned>(ctas), kThreads, smem, stream>>>(tq, tk, tv, p);
   return cudaGetLastError();
 }

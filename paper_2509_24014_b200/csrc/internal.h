@@ -47,6 +47,8 @@ struct AttnParams {
   int group;               // heads_q / heads_kv
   int num_q_tiles;         // 128-row query tiles per (batch, head)
   int num_blocks;          // sparse only: pattern blocks per row (seq_len / block_size)
+  int num_items;           // batch * heads_q * num_q_tiles: 128-row query tiles in all
+  int max_ctas;            // > 0: launch at most this many CTAs and let each run through several items
   float scale_log2;        // softmax scale * log2(e)
   const int32_t* row_ptr;  // sparse only
   const int32_t* col_idx;  // sparse only
