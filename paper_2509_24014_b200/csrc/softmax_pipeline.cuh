@@ -141,8 +141,9 @@ struct RowStatWriter {
         carry = s;
         carry_m = m;
       } else {
-        // the even half was summed against carry_m <= m: bring it to the current reference
-        const float both = s + carry * fast_exp2(carry_m - m);
+        // the even half was summed against carry_m <= m: bring it to the current reference (the two
+        // are equal unless the maximum moved between the two halves, which is rare)
+        const float both = (carry_m == m) ? s + carry : s + carry * fast_exp2(carry_m - m);
         __stcs(dst + static_cast<int64_t>(g64 >> 1) * 128, m + __log2f(both));
       }
     }

@@ -179,3 +179,44 @@ def test_token_major_layout_through_every_entry_point():
     torch.cuda.synchronize()
     check_outputs(o_sp, orc.attn_sparse(qd, kd, vd, rp, ci, bs), "token-major sparse")
     assert sd.sparsed_last_device_status(ws) == (0, 0)
+
+
+def test_ctas_that_run_through_several_query_tiles_match_one_tile_per_cta():
+    """Block-sparse launches with more query tiles than CTAs fit on the device let every CTA roll on into
+    further tiles (ring slots, S buffers and barrier phases carry over). 768 query tiles with ragged
+    user-built lists, empty ones among them, must give bitwise what the same heads give when launched one
+    head at a time (64 tiles each: one tile per CTA), and agree with the oracle on sampled rows."""
+    B, Hq, Hkv, L, bs = 1, 12, 4, 8192, 128
+    cfg = syn.AttnConfig("roll", B, Hq, Hkv, L, 128, bs, 0.1, 0, seed=404, plant_norm=6.0)
+    q, k, v = syn.make_qkv(cfg, DEV)
+    nb = L // bs
+    rng = np.random.default_rng(404)
+    lists = []
+    for r in range(Hq * nb):
+        n = int(rng.integers(0, 7)) if r % 5 else 0             # every fifth list is empty
+        lists.append(sorted(rng.choice(nb, size=n, replace=False).tolist()))
+    rp = np.cumsum([0] + [len(x) for x in lists]).astype(np.int32)
+    ci = np.concatenate([np.asarray(x, dtype=np.int32) for x in lists] + [np.zeros(1, np.int32)]).astype(np.int32)
+    rp_d, ci_d = torch.from_numpy(rp).to(DEV), torch.from_numpy(ci).to(DEV)
+    ws = sd.new_workspace(256, DEV)
+    o_all = torch.full_like(q, float("nan"))
+    sd.sparsed_attn_sparse(q, k, v, o_all, sd.pattern_from_csr(rp_d, ci_d, bs, nb, B, Hq), ws)
+    o_one = torch.full_like(q, float("nan"))
+    group = Hq // Hkv
+    for h in range(Hq):
+        rp_h = (rp_d[h * nb:(h + 1) * nb + 1]).contiguous()   # absolute offsets into the shared col_idx
+        pat_h = sd.pattern_from_csr(rp_h, ci_d, bs, nb, 1, 1)
+        sd.sparsed_attn_sparse(q[:, h:h + 1], k[:, h // group:h // group + 1], v[:, h // group:h // group + 1],
+                               o_one[:, h:h + 1], pat_h, ws)
+    torch.cuda.synchronize()
+    assert sd.sparsed_last_device_status(ws) == (0, 0)
+    assert torch.equal(o_all, o_one)
+    for h, ib in ((0, 0), (3, 17), (7, 63), (11, 40), (5, 5)):
+        r = h * nb + ib
+        rows = slice(ib * bs, (ib + 1) * bs)
+        if not lists[r]:
+            assert torch.all(o_all[0, h, rows] == 0)
+        else:
+            ref = orc.head_sparse_rows(to_f64(q[0, h]), to_f64(k[0, h // group]), to_f64(v[0, h // group]), ib,
+                                       lists[r], bs)
+            check_outputs(o_all[0, h, rows], ref, f"rolled-on tile h{h} ib{ib}")
