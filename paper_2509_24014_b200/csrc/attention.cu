@@ -78,11 +78,14 @@ struct AttnSmem {
 };
 
 // kDense: walk every key tile of the sequence (kBlock must be 128 then; no block lists are read).
-template <int kBlock, bool kDense>
+// kMultiItem: a CTA may be given several query tiles (launched with fewer CTAs than tiles); without it the
+// item loops below run once and their running counters fold to zero at compile time.
+template <int kBlock, bool kDense, bool kMultiItem>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
   static_assert(!kDense || kBlock == 128, "the dense walk uses the unpacked layout");
+  static_assert(!kMultiItem || kBlock == 128, "the packed walk prepares its union once per CTA");
   using Smem = AttnSmem<kBlock>;
   constexpr bool kPacked = Smem::kPacked;
   constexpr int kSlots = Smem::kSlots;
@@ -347,6 +350,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         issue_load(cur, slot, i & 1, kv_row0, kv_row1, blocks_here);
         TL(22);
       }
+      if constexpr (!kMultiItem) break;
       load0 += 2 * num_tiles;
       if (num_tiles > 0) prev_tiles = num_tiles;
     }
@@ -363,7 +367,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     for (int item = first_item; ok && item < n_items; item += gridDim.x) {
       if (item != first_item) cur = describe(item);
       const int num_tiles = tiles_of(cur);
-      if (num_tiles == 0) continue;
+      if (num_tiles == 0) {
+        if constexpr (!kMultiItem) break;
+        continue;
+      }
       // S_t = Q K_t^T into S buffer (tile0 + t) & 1
       auto issue_qk = [&](int t) -> bool {
         const int g = load0 + 2 * t;
@@ -402,6 +409,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         issue_pv64(tO, tmem + kColS + (gt & 1) * kTileN, v_lo0 + slot * slot_step, t > 0, &sm.done[slot]);
         TL(15);
       }
+      if constexpr (!kMultiItem) break;
       load0 += 2 * num_tiles;
       tile0 += num_tiles;
     }
@@ -532,6 +540,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (p.lse != nullptr && row_valid)
           p.lse[static_cast<int64_t>(cur.bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
       }
+      if constexpr (!kMultiItem) break;
       tc_fence_before();   // the next item's first P V overwrites O: order these reads before its hand-over
       load0 += 2 * num_tiles;
       tile0 += num_tiles;
@@ -547,19 +556,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int kBlock, bool kDense>
+template <int kBlock, bool kDense, bool kMultiItem>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kBlock, kDense>;
+  auto kernel = attn_kernel<kBlock, kDense, kMultiItem>;
   const int smem = static_cast<int>(sizeof(AttnSmem<kBlock>));
   static SmemLimit limit;  // per template instantiation
   cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
   if (e != cudaSuccess) return e;
-  // one CTA per item, or (p.max_ctas > 0; not for the packed walk, which prepares its union once per CTA)
-  // at most that many CTAs, each running through its share of the items
+  // one CTA per item, or (kMultiItem and p.max_ctas > 0) at most that many CTAs, each running through its
+  // share of the items
   long long ctas = p.num_items;
   if (ctas <= 0) return cudaSuccess;
-  if (kBlock == kTileM && p.max_ctas > 0 && ctas > p.max_ctas) ctas = p.max_ctas;
+  if (kMultiItem && p.max_ctas > 0 && ctas > p.max_ctas) ctas = p.max_ctas;
   kernel<<<static_cast<unsigned>(ctas), kThreads, smem, stream>>>(tq, tk, tv, p);
   return cudaGetLastError();
 }
@@ -572,15 +581,15 @@ int attn_sparse_max_blocks(int block_size) { return block_size < kTileM ? kMaxPa
 // p.num_q_tiles = ceil(seq_len / 128), p.num_blocks = seq_len / block_size.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128, false>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<64, false>(tq, tk, tv, p, batch, stream);
-  return launch<32, false>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<128, false, true>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<64, false, false>(tq, tk, tv, p, batch, stream);
+  return launch<32, false, false>(tq, tk, tv, p, batch, stream);
 }
 
 // Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream) {
-  return launch<128, true>(tq, tk, tv, p, batch, stream);
+  return launch<128, true, false>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed
