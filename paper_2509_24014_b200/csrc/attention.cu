@@ -32,6 +32,8 @@
 //     its own query block did not keep; a tile in which a warp keeps nothing costs it no
 //     exponentials. All 128 rows of every MMA belong to real queries, and neighbouring query blocks
 //     share the K/V tiles they have in common.
+#include <type_traits>
+
 #include "internal.h"
 #include "softmax_pipeline.cuh"
 
@@ -80,12 +82,14 @@ struct AttnSmem {
 // kDense: walk every key tile of the sequence (kBlock must be 128 then; no block lists are read).
 // kMultiItem: a CTA may be given several query tiles (launched with fewer CTAs than tiles); without it the
 // item loops below run once and their running counters fold to zero at compile time.
-template <int kBlock, bool kDense, bool kMultiItem>
+// kStatKeys: dense only: 0, or record one row statistic per 32 / 64 / 128 keys.
+template <int kBlock, bool kDense, bool kMultiItem, int kStatKeys>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
   static_assert(!kDense || kBlock == 128, "the dense walk uses the unpacked layout");
   static_assert(!kMultiItem || kBlock == 128, "the packed walk prepares its union once per CTA");
+  static_assert(kDense || kStatKeys == 0, "row statistics are recorded by the dense walk only");
   using Smem = AttnSmem<kBlock>;
   constexpr bool kPacked = Smem::kPacked;
   constexpr int kSlots = Smem::kSlots;
@@ -428,26 +432,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int num_tiles = tiles_of(cur);
       const bool group_valid = my_group < cur.groups_here;
       RowState st{-INFINITY, 0.f};
-      RowStatWriter stats;
-      if constexpr (kDense) {
-        const int groups = (p.seq_len + p.stat_keys - 1) / p.stat_keys;
+      RowStatWriter<kStatKeys> stats;
+      if constexpr (kStatKeys > 0) {
+        const int groups = (p.seq_len + kStatKeys - 1) / kStatKeys;
         float* first = nullptr;
         if (p.tile_lse != nullptr && cur.q_row0 + tid < p.seq_len)
           first = p.tile_lse + (static_cast<int64_t>(cur.bh) * p.num_q_tiles + cur.q_tile) * groups * kTileM + tid;
-        stats.init(first, p.stat_keys, groups);
+        stats.init(first, groups);
       }
-      for (int t = 0; t < num_tiles; ++t) {
+      // One 64-key tile of the softmax. kOdd (a compile-time tag) is only used by the walk that records one
+      // statistic per 128 keys: it runs its tiles in pairs so that the even / odd halves of a statistic are
+      // resolved at compile time instead of costing the busiest warps of the kernel instructions per tile
+      // (pairing every walk was measured too: it costs registers and 2.5 % of the plain dense pass).
+      auto tile_body = [&](int t, auto odd_tag) -> bool {
+        constexpr bool kOdd = decltype(odd_tag)::value;
         TL(1);
         // S_t is ready when the Q K^T batch that read ring load 2t of this item has completed
         const int gk = load0 + 2 * t;
-        if (!mbar_wait(&sm.done[gk % kSlots], (gk / kSlots) & 1, &sm.abort_flag, p.status, 30)) {
-          ok = false;
-          break;
-        }
+        if (!mbar_wait(&sm.done[gk % kSlots], (gk / kSlots) & 1, &sm.abort_flag, p.status, 30)) return false;
         TL(2);
         tc_fence_after();
-        const int gt = tile0 + t;
-        const uint32_t tS = tmem + kColS + (gt & 1) * kTileN + lane_base;
+        const int buf = (tile0 + t) & 1;   // S buffer of the tile
+        const uint32_t tS = tmem + kColS + buf * kTileN + lane_base;
         // packed walk: which 32-column chunks of this tile hold key blocks this warp's query block kept
         bool keep0 = true, keep1 = true;
         if constexpr (kPacked) {
@@ -465,7 +471,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
         }
         uint32_t pk[32];
-        float2 stat_sums = make_float2(0.f, 0.f);
         if (kPacked && !keep0 && !keep1) {
           // nothing of this tile is kept by this warp's query block: P = 0, no exponentials
 #pragma unroll
@@ -501,26 +506,31 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             if (t > 0) {
               // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring load 2t-1) has drained
               const int gp = load0 + 2 * (t - 1) + 1;
-              if (!mbar_wait(&sm.done[gp % kSlots], (gp / kSlots) & 1, &sm.abort_flag, p.status, 32)) {
-                ok = false;
-                break;
-              }
+              if (!mbar_wait(&sm.done[gp % kSlots], (gp / kSlots) & 1, &sm.abort_flag, p.status, 32)) return false;
               tc_fence_after();
               rescale_accumulator_row(tO + lane_base, alpha);
               if (p.slow_path_events != nullptr && lane == 0) atomicAdd(p.slow_path_events, 1ull);
             }
           }
           st.l += sums.x + sums.y;
-          stat_sums = sums;
+          if constexpr (kStatKeys > 0) stats.template begin<kOdd>(sums, st.m);
         }
         TL(4);
         tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&sm.p_full[gt & 1]);
+        mbar_arrive(&sm.p_full[buf]);
         TL(5);
-        // the statistic is worked out after P has been handed over: off the S -> P -> P V chain
-        if constexpr (kDense) stats.put(t, stat_sums, st.m);
+        // the statistic is stored after P has been handed over: off the S -> P -> P V chain
+        if constexpr (kStatKeys > 0) stats.template finish<kOdd>(st.m);
+        return true;
+      };
+      if constexpr (kStatKeys == 128) {
+        int t = 0;
+        for (; ok && t + 1 < num_tiles; t += 2) ok = tile_body(t, std::false_type{}) && tile_body(t + 1, std::true_type{});
+        if (ok && t < num_tiles) ok = tile_body(t, std::false_type{});
+      } else {
+        for (int t = 0; ok && t < num_tiles; ++t) ok = tile_body(t, std::false_type{});
       }
       if (!ok) break;
 
@@ -556,10 +566,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int kBlock, bool kDense, bool kMultiItem>
+template <int kBlock, bool kDense, bool kMultiItem, int kStatKeys>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kBlock, kDense, kMultiItem>;
+  auto kernel = attn_kernel<kBlock, kDense, kMultiItem, kStatKeys>;
   const int smem = static_cast<int>(sizeof(AttnSmem<kBlock>));
   static SmemLimit limit;  // per template instantiation
   cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
@@ -581,15 +591,18 @@ int attn_sparse_max_blocks(int block_size) { return block_size < kTileM ? kMaxPa
 // p.num_q_tiles = ceil(seq_len / 128), p.num_blocks = seq_len / block_size.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128, false, true>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<64, false, false>(tq, tk, tv, p, batch, stream);
-  return launch<32, false, false>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<128, false, true, 0>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<64, false, false, 0>(tq, tk, tv, p, batch, stream);
+  return launch<32, false, false, 0>(tq, tk, tv, p, batch, stream);
 }
 
 // Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream) {
-  return launch<128, true, false>(tq, tk, tv, p, batch, stream);
+  if (p.tile_lse == nullptr) return launch<128, true, false, 0>(tq, tk, tv, p, batch, stream);
+  if (p.stat_keys == 128) return launch<128, true, false, 128>(tq, tk, tv, p, batch, stream);
+  if (p.stat_keys == 64) return launch<128, true, false, 64>(tq, tk, tv, p, batch, stream);
+  return launch<128, true, false, 32>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed

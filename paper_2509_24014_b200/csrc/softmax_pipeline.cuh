@@ -112,39 +112,63 @@ __device__ __forceinline__ void rescale_accumulator_row(uint32_t t_acc_row, floa
 // [key group][row in tile] so that a query tile's statistics are one contiguous run. The
 // attention kernels feed it 64 keys at a time (the two 32-column sums of a softmax group,
 // relative to the reference maximum in use at that moment).
+template <int kStatKeys>   // 0 = no statistics, else 32, 64 or 128 keys per statistic
 struct RowStatWriter {
-  float* dst;        // first statistic of this row: + (query tile * groups) * 128 + row in tile; null = off
-  int stat_keys;
-  int groups;        // key groups per row = ceil(seq_len / stat_keys)
+  float* next;       // where this row's next statistic goes (statistics of one row are 128 floats apart)
+  int left;          // statistics still to be written for this row (0 for rows beyond the sequence end)
   float carry;       // 128-key groups: sum of the even 64-key half, relative to carry_m
   float carry_m;
+  float lg0, lg1;    // log2 of the sums of the group in flight (begin -> finish)
 
-  __device__ __forceinline__ void init(float* first, int keys, int n_groups) {
-    dst = first;
-    stat_keys = keys;
-    groups = n_groups;
+  // first: the row's first statistic, or null for a row beyond the sequence end; n_groups = ceil(seq_len / kStatKeys)
+  __device__ __forceinline__ void init(float* first, int n_groups) {
+    next = first;
+    left = first != nullptr ? n_groups : 0;
     carry = 0.f;
     carry_m = 0.f;
+    lg0 = lg1 = 0.f;
   }
-  // g64: index of the 64-key group within the row; sums: its two 32-column sums relative to m.
-  __device__ __forceinline__ void put(int g64, float2 sums, float m) {
-    if (dst == nullptr) return;
-    // (a 64-key group can lie wholly beyond a ragged sequence end: it has no statistic)
-    if (stat_keys == 64) {
-      if (g64 < groups) __stcs(dst + static_cast<int64_t>(g64) * 128, m + __log2f(sums.x + sums.y));
-    } else if (stat_keys == 32) {
-      if (2 * g64 < groups) __stcs(dst + static_cast<int64_t>(2 * g64) * 128, m + __log2f(sums.x));
-      if (2 * g64 + 1 < groups) __stcs(dst + static_cast<int64_t>(2 * g64 + 1) * 128, m + __log2f(sums.y));
-    } else {
+  // Two halves, because a warp issues in order: `begin` only STARTS the logarithm(s) as soon as the sums
+  // exist; `finish`, called after P has been handed over (by then the results are there), adds the
+  // reference maximum and stores. Every instruction here is paid by the softmax warps, the busiest
+  // warps of the kernel (recording costs 5-10 % of the dense pass), hence the running pointer and counter
+  // instead of index arithmetic.
+  // kOdd: this is the second 64-key tile of a 128-key group; sums: the tile's two 32-column sums relative to m.
+  template <bool kOdd>
+  __device__ __forceinline__ void begin(float2 sums, float m) {
+    if constexpr (kStatKeys == 64) {
+      lg0 = fast_log2(sums.x + sums.y);
+    } else if constexpr (kStatKeys == 32) {
+      lg0 = fast_log2(sums.x);
+      lg1 = fast_log2(sums.y);
+    } else if constexpr (kStatKeys == 128) {
       const float s = sums.x + sums.y;
-      if ((g64 & 1) == 0) {
+      if constexpr (!kOdd) {
         carry = s;
         carry_m = m;
       } else {
-        // the even half was summed against carry_m <= m: bring it to the current reference (the two
-        // are equal unless the maximum moved between the two halves, which is rare)
-        const float both = (carry_m == m) ? s + carry : s + carry * fast_exp2(carry_m - m);
-        __stcs(dst + static_cast<int64_t>(g64 >> 1) * 128, m + __log2f(both));
+        // the even half was summed against carry_m <= m: bring it to the current reference
+        lg0 = fast_log2(fmaf(carry, fast_exp2(carry_m - m), s));
+      }
+    }
+  }
+  // (a group that lies wholly beyond a ragged sequence end has no statistic: `left` runs out first)
+  template <bool kOdd>
+  __device__ __forceinline__ void finish(float m) {
+    if constexpr (kStatKeys == 64) {
+      if (left > 0) __stcs(next, m + lg0);
+      next += 128;
+      --left;
+    } else if constexpr (kStatKeys == 32) {
+      if (left > 0) __stcs(next, m + lg0);
+      if (left > 1) __stcs(next + 128, m + lg1);
+      next += 256;
+      left -= 2;
+    } else if constexpr (kStatKeys == 128) {
+      if constexpr (kOdd) {
+        if (left > 0) __stcs(next, m + lg0);
+        next += 128;
+        --left;
       }
     }
   }
