@@ -43,33 +43,40 @@ METRIC = "block-sparse attn TFLOP/s, % bf16 peak, speedup vs own dense kernel at
 # since is reported as null with the reason, instead of going stale silently.
 _C2_ATTN = "ncu --set full capture of one launch on the 8k workload (summary under profiles/)"
 _C2_POOL = "ncu --set full capture of one launch on the 8k workload (summary under profiles/)"
-_ATTN_SRC, _ATTN_SHA = "paper_2509_24014_b200/csrc/attention.cu", "08fa8b826bec"
-_POOL_SRC, _POOL_SHA = "paper_2509_24014_b200/csrc/pool_select.cu", "840b284c40be"
+_ATTN_SRC = ("paper_2509_24014_b200/csrc/attention.cu", "paper_2509_24014_b200/csrc/softmax_pipeline.cuh",
+             "paper_2509_24014_b200/csrc/sm100_primitives.cuh")
+_ATTN_SHA = "ac42ce860f5a"
+_POOL_SRC = ("paper_2509_24014_b200/csrc/pool_select.cu", "paper_2509_24014_b200/csrc/topk_device.cuh")
+_POOL_SHA = "2a48dbebbbc2"
 NCU_DRAM_TRAFFIC = {
-    ("attn_kernel<dense>", "c2"): (201476096 + 100872448, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
-    ("attn_kernel<sparse>", "c2"): (156410112 + 42415616, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
-    ("pool_select_kernel", "c2"): (68195328 + 522496, _C2_POOL, _POOL_SRC, _POOL_SHA),
+    ("attn_kernel<dense>", "c2"): (201754368 + 105816064, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
+    ("attn_kernel<sparse>", "c2"): (156551680 + 43603712, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
+    ("pool_select_kernel", "c2"): (68194816 + 587776, _C2_POOL, _POOL_SRC, _POOL_SHA),
     # 64k workload: the 8k capture scaled by the algorithmic bytes of a launch (traffic was the algorithmic
     # traffic at 8k: every K/V re-read hits L2), instead of a multi-counter capture of a 7 GB workload.
     # dense + statistics: Q,K,V,O + LSE + statistics = 6450 MB at 64k against 336 MB at 8k
-    ("attn_kernel<dense>", "c4"): (int((201476096 + 100872448) * 6450.0 / 336.0), _C2_ATTN + ", scaled x19.2 by algorithmic bytes",
+    ("attn_kernel<dense>", "c4"): (int((201754368 + 105816064) * 6450.0 / 336.0), _C2_ATTN + ", scaled x19.2 by algorithmic bytes",
                                    _ATTN_SRC, _ATTN_SHA),
     # sparse: Q + O + touched K,V: 8x the rows and 8x the K/V of the 8k workload
-    ("attn_kernel<sparse>", "c4"): ((156410112 + 42415616) * 8, _C2_ATTN + ", scaled x8 by algorithmic bytes",
+    ("attn_kernel<sparse>", "c4"): ((156551680 + 43603712) * 8, _C2_ATTN + ", scaled x8 by algorithmic bytes",
                                     _ATTN_SRC, _ATTN_SHA),
     # pooling: the statistics stream, 64x the 8k one (rows x8, key blocks x8)
-    ("pool_select_kernel", "c4"): ((68195328 + 522496) * 64, _C2_POOL + ", scaled x64 by algorithmic bytes",
+    ("pool_select_kernel", "c4"): ((68194816 + 587776) * 64, _C2_POOL + ", scaled x64 by algorithmic bytes",
                                    _POOL_SRC, _POOL_SHA),
 }
 
 
-def _source_digest(rel_path):
+def _source_digest(rel_paths):
+    """sha256 prefix over the named source files (a kernel may be spread over several)."""
     import hashlib
+    h = hashlib.sha256()
     try:
-        with open(os.path.join(ROOT, rel_path), "rb") as f:
-            return hashlib.sha256(f.read()).hexdigest()[:12]
+        for rel in rel_paths:
+            with open(os.path.join(ROOT, rel), "rb") as f:
+                h.update(f.read())
     except OSError:
         return None
+    return h.hexdigest()[:12]
 
 
 def ncu_traffic(kernel, workload):
@@ -79,7 +86,7 @@ def ncu_traffic(kernel, workload):
         return None, "no ncu capture for this kernel and workload"
     nbytes, where, src, digest = rec
     if _source_digest(src) != digest:
-        return None, f"stale: {src} changed since the capture ({where})"
+        return None, f"stale: {' / '.join(src)} changed since the capture ({where})"
     return nbytes, where
 
 
