@@ -277,11 +277,23 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": workload_name(cfg), "timing": "host perf_counter"},
+            "data": "synthetic", "config": bench_config(cfg, k_pre, k_gen, args.gpus), "timing": "host perf_counter",
             "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+def bench_config(cfg, k_pre, k_gen, world=1, shard_heads=False):
+    """The `config` object of the JSON line; the same for this library's arm and the reference arm."""
+    nb = cfg.num_blocks
+    nnz = cfg.batch * cfg.heads_q * nb * (k_pre + k_gen)
+    qkvo_gb = 2.0 * cfg.batch * cfg.seq_len * cfg.head_dim * (2 * cfg.heads_q + 2 * cfg.heads_kv) / 1e9
+    return {"workload": workload_name(cfg), "step": "attn_full_stats -> select_from_stats -> attn_sparse",
+            "kept_per_row": [k_pre, k_gen], "nnz": nnz, "density": nnz / (cfg.batch * cfg.heads_q * nb * nb),
+            "l2": "inputs larger than L2 (Q,K,V,O = %.2f GB per pass)" % qkvo_gb,
+            "parallelism": ("heads sharded over ranks, no collective" if shard_heads else
+                            "replicas only" if world > 1 else "single GPU")}
 
 
 def workload_name(cfg):
@@ -654,11 +666,7 @@ def run_ours(args, cfg):
         "ms_per_step": total_ms / n, "higher_is_better": True, "scaling": "strong" if shard_heads else "weak",
         "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "step": "attn_full_stats -> select_from_stats -> attn_sparse",
-                   "kept_per_row": [k_pre, k_gen], "nnz": nnz, "density": nnz / (B * Hq * nb * nb),
-                   "l2": "inputs larger than L2 (Q,K,V,O = %.2f GB per pass)" % qkvo_gb,
-                   "parallelism": ("heads sharded over ranks, no collective" if shard_heads else
-                                   "replicas only" if world > 1 else "single GPU")},
+        "config": bench_config(cfg, k_pre, k_gen, world, shard_heads),
         "pct_bf16_peak": 100.0 * per_gpu_sparse / peak,
         "pct_bf16_peak_sustained": 100.0 * per_gpu_sparse / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
         "pct_bf16_nominal_2250": 100.0 * per_gpu_sparse / 2250.0,
