@@ -15,9 +15,9 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 OBJ_DIR = os.path.join(PKG_DIR, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libsparsed.so")
-SOURCES = ["api.cu", "attention.cu", "scoring.cu", "topk.cu", "pool_select.cu", "patterns.cu",
+SOURCES = ["api.cu", "attention.cu", "attention_dense_pair.cu", "scoring.cu", "topk.cu", "pool_select.cu", "patterns.cu",
            "pooled_qk.cu"]
-HEADERS = ["internal.h", "sm100_primitives.cuh", "softmax_pipeline.cuh", "topk_device.cuh",
+HEADERS = ["internal.h", "sm100_primitives.cuh", "sm100_pair_primitives.cuh", "softmax_pipeline.cuh", "topk_device.cuh",
            os.path.join("..", "..", "include", "sparsed.h")]
 ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC"]

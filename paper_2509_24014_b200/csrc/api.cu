@@ -2,6 +2,7 @@
 // workspace layout and kernel dispatch. Declarations and contracts are in sparsed.h.
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -351,6 +352,15 @@ sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stre
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
+// Which dense kernel runs: the CTA-pair one when the environment says SPARSED_DENSE_KERNEL=pair (read once).
+static bool dense_pair_kernel() {
+  static const bool pair = [] {
+    const char* v = std::getenv("SPARSED_DENSE_KERNEL");
+    return v != nullptr && std::strcmp(v, "pair") == 0;
+  }();
+  return pair;
+}
+
 static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
                                      float* lse_or_null, float* tile_lse_or_null, int stat_keys, void* ws,
                                      size_t ws_bytes, void* cuda_stream) {
@@ -362,11 +372,11 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   if (!aligned16(lse_or_null) || !aligned16(tile_lse_or_null)) return SPARSED_ERR_ALIGNMENT;
   if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
-  const int kv_box_rows = 64;
+  const bool pair = dense_pair_kernel();
   CUtensorMap tq, tk, tv;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, kv_box_rows)) != SPARSED_OK) return st;
-  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, kv_box_rows)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, pair ? 32 : 64)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 64)) != SPARSED_OK) return st;
   AttnParams p;
   p.o = o;
   p.o_stride_b = rs.o[0];
@@ -388,7 +398,8 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   p.col_idx = nullptr;
   p.col_capacity = 0;
   p.status = static_cast<DeviceStatus*>(ws);
-  cudaError_t e = launch_attn_dense(tq, tk, tv, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = pair ? launch_attn_dense_pair(tq, tk, tv, p, static_cast<cudaStream_t>(cuda_stream))
+                      : launch_attn_dense(tq, tk, tv, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 

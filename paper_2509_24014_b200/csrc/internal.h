@@ -121,6 +121,9 @@ size_t pooled_qk_means_bytes(int batch, int heads_q, int heads_kv, int nb);
 cudaError_t launch_pooled_qk_select(const PooledQkParams& p, cudaStream_t stream);
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream);
+// The same pass with the MMAs spanning CTA pairs (cta_group::2); K tensor map with 32-row boxes.
+cudaError_t launch_attn_dense_pair(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                   const AttnParams& p, cudaStream_t stream);
 int attn_sparse_max_blocks(int block_size);   // most key blocks per row the sparse kernel handles
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream);
