@@ -145,6 +145,9 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
  *                               recorded with.
  * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; the selection needs
  * seq_len / block_size <= 2048 (UNSUPPORTED beyond). Both buffers are caller-owned device memory.
+ * sparsed_attn_full_stats runs on a kernel of its own (MMAs spanning pairs of CTAs, launched as
+ * clusters of two); the environment variable SPARSED_DENSE_KERNEL=single|pair, read at the first call,
+ * sends both dense entry points to one kernel, for measurements.
  */
 sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, int32_t block_size,
                                         size_t *out_bytes); /* host only */
@@ -279,8 +282,9 @@ sparsed_status sparsed_pattern_validate(const sparsed_pattern *pattern, void *ws
 
 /* Reads the device status word (synchronises the stream). code 0 = fine, 1 = a bounded wait ran out
  * (`where` identifies the wait), 2 = a kernel found its shared memory misaligned, 3 = sparsed_attn_sparse
- * met a row_ptr entry that points outside col_idx (that query block's rows were written as zeros).
- * Returns SPARSED_ERR_DEVICE_TIMEOUT if code != 0. */
+ * met a row_ptr entry that points outside col_idx (that query block's rows were written as zeros),
+ * 4 = the two CTAs of a pair in sparsed_attn_full_stats got different tensor-memory bases (the pair did no
+ * work). Returns SPARSED_ERR_DEVICE_TIMEOUT if code != 0. */
 sparsed_status sparsed_last_device_status(void *ws, void *cuda_stream, int32_t *code, int32_t *where);
 
 /*

@@ -352,13 +352,18 @@ sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stre
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
-// Which dense kernel runs: the CTA-pair one when the environment says SPARSED_DENSE_KERNEL=pair (read once).
-static bool dense_pair_kernel() {
-  static const bool pair = [] {
+// Which dense kernel runs. The pass that also records row statistics goes to the kernel whose MMAs span CTA
+// pairs (its softmax warps have the slack to record them for free: measured 2-5 % faster from 8k to 64k); the
+// plain pass stays on the single-CTA kernel (equal under sustained load, faster on short launches). The
+// environment variable SPARSED_DENSE_KERNEL=pair|single (read once) forces one of them, for A/B measurements.
+static bool dense_pair_kernel(bool with_stats) {
+  static const int forced = [] {
     const char* v = std::getenv("SPARSED_DENSE_KERNEL");
-    return v != nullptr && std::strcmp(v, "pair") == 0;
+    if (v != nullptr && std::strcmp(v, "pair") == 0) return 1;
+    if (v != nullptr && std::strcmp(v, "single") == 0) return 0;
+    return -1;
   }();
-  return pair;
+  return forced >= 0 ? forced == 1 : with_stats;
 }
 
 static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
@@ -372,7 +377,7 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   if (!aligned16(lse_or_null) || !aligned16(tile_lse_or_null)) return SPARSED_ERR_ALIGNMENT;
   if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
-  const bool pair = dense_pair_kernel();
+  const bool pair = dense_pair_kernel(tile_lse_or_null != nullptr);
   CUtensorMap tq, tk, tv;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
   if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, pair ? 32 : 64)) != SPARSED_OK) return st;

@@ -36,7 +36,7 @@ constexpr int kHeadDim = 128;
 constexpr int kTileM = 128;        // query rows per CTA and stream
 constexpr int kTileN = 64;         // keys per pipeline step
 constexpr int kStreams = 2;
-constexpr int kSlots = 8;          // 8 KB ring slots per stream: half a K tile or half a V tile each
+constexpr int kSlots = 20;         // 8 KB ring slots (half a K tile or half a V tile each), shared by both streams
 constexpr int kThreads = 384;      // warps 0-3 / 4-7: softmax of stream 0 / 1; 8, 9: producers; 10, 11: issuers
 constexpr int kTmemCols = 512;     // per stream 256: two S buffers of 64 columns, then O (128)
 constexpr int kColS = 0;
@@ -45,15 +45,17 @@ constexpr int kArrivalsP = 8;      // four softmax warps in each CTA of the pair
 
 struct PairStream {
   alignas(1024) __nv_bfloat16 q[2][kTileM * 64];      // two 64-wide halves of head_dim
-  // K half-tile: two [32 keys x 64] halves of head_dim (4 KB each); V half-tile: [64 keys x 64 columns of head_dim]
-  alignas(1024) __nv_bfloat16 kv[kSlots][kTileN * 64];
-  uint64_t q_full, kv_full[kSlots];   // used in the leader CTA: bytes of both CTAs
-  uint64_t done[kSlots];              // in both CTAs: the MMAs that read the slot have completed
+  uint64_t q_full;                    // used in the leader CTA: bytes of both CTAs
+  uint64_t done[kSlots];              // in both CTAs: this stream's MMAs that read the slot have completed
   uint64_t p_full[2];                 // used in the leader CTA: P of both CTAs is in tensor memory
 };
 
 struct PairSmem {
+  // K half-tile: two [32 keys x 64] halves of head_dim (4 KB each); V half-tile: [64 keys x 64 columns of head_dim].
+  // Both streams (neighbouring query tiles of one head) read every tile from the same slot.
+  alignas(1024) __nv_bfloat16 kv[kSlots][kTileN * 64];
   PairStream stream[kStreams];
+  uint64_t kv_full[kSlots];           // used in the leader CTA: bytes of both CTAs
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -99,13 +101,11 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     for (int s = 0; s < kStreams; ++s) {
       PairStream& S = sm.stream[s];
       mbar_init(&S.q_full, 1);
-      for (int i = 0; i < kSlots; ++i) {
-        mbar_init(&S.kv_full[i], 1);
-        mbar_init(&S.done[i], 1);
-      }
+      for (int i = 0; i < kSlots; ++i) mbar_init(&S.done[i], 1);
       mbar_init(&S.p_full[0], kArrivalsP);
       mbar_init(&S.p_full[1], kArrivalsP);
     }
+    for (int i = 0; i < kSlots; ++i) mbar_init(&sm.kv_full[i], 1);
     sm.abort_flag = 0;
     mbar_fence_init();
   }
@@ -147,36 +147,47 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
   if (!active) {
     // nothing to do for this warp
-  } else if (warp == 8 || warp == 9) {
-    // =============================== TMA producer ============================================
-    const uint32_t q_full_leader = map_to_cta(smem_u32(&S.q_full), 0);
+  } else if (warp == 9) {
+    // (spare warp)
+  } else if (warp == 8) {
+    // =============================== TMA producer (both streams) =============================
+    const bool two = pair_ok && (first_tile + 2) < p.num_q_tiles;   // stream 1 has rows
     if (elect_one_sync()) {
-      if (rank == 0) mbar_expect_tx(&S.q_full, 2 * kTileM * kHeadDim * 2);   // rows beyond the sequence arrive as zeros
-      tma_load_4d_pair(S.q[0], &tm_q, q_full_leader, 0, q_row0, head, batch);
-      tma_load_4d_pair(S.q[1], &tm_q, q_full_leader, 64, q_row0, head, batch);
+      for (int s = 0; s < (two ? 2 : 1); ++s) {
+        PairStream& T = sm.stream[s];
+        const uint32_t q_full_leader = map_to_cta(smem_u32(&T.q_full), 0);
+        const int row0 = (first_tile + 2 * s + static_cast<int>(rank)) * kTileM;
+        if (rank == 0) mbar_expect_tx(&T.q_full, 2 * kTileM * kHeadDim * 2);   // rows beyond the sequence arrive as zeros
+        tma_load_4d_pair(T.q[0], &tm_q, q_full_leader, 0, row0, head, batch);
+        tma_load_4d_pair(T.q[1], &tm_q, q_full_leader, 64, row0, head, batch);
+      }
     }
     __syncwarp();
     bool ok = true;
-    // load i: this CTA's half of K (even) or V (odd) of tile i / 2
+    // load i: this CTA's half of K (even) or V (odd) of tile i / 2, for both streams
     for (int i = 0; ok && i < 2 * num_tiles; ++i) {
       const int slot = i % kSlots;
       if (i >= kSlots) {
-        ok = mbar_wait(&S.done[slot], ((i / kSlots) - 1) & 1, &sm.abort_flag, p.status, 40);
+        // free once the MMAs of every stream that read it have completed
+        const uint32_t parity = ((i / kSlots) - 1) & 1;
+        ok = two ? mbar_wait2(&sm.stream[0].done[slot], parity, &sm.stream[1].done[slot], parity, &sm.abort_flag,
+                              p.status, 40)
+                 : mbar_wait(&sm.stream[0].done[slot], parity, &sm.abort_flag, p.status, 40);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
       if (elect_one_sync()) {
-        const uint32_t full_leader = map_to_cta(smem_u32(&S.kv_full[slot]), 0);
-        if (rank == 0) mbar_expect_tx(&S.kv_full[slot], 2 * kTileN * 64 * 2);   // both CTAs' halves
+        const uint32_t full_leader = map_to_cta(smem_u32(&sm.kv_full[slot]), 0);
+        if (rank == 0) mbar_expect_tx(&sm.kv_full[slot], 2 * kTileN * 64 * 2);   // both CTAs' halves
         const int key0 = (i >> 1) * kTileN;
         if ((i & 1) == 0) {
           // keys [32 rank, 32 rank + 32) of the tile, all of head_dim
-          tma_load_4d_pair(S.kv[slot], &tm_k, full_leader, 0, key0 + 32 * static_cast<int>(rank), kv_head, batch);
-          tma_load_4d_pair(S.kv[slot] + 32 * 64, &tm_k, full_leader, 64, key0 + 32 * static_cast<int>(rank), kv_head,
+          tma_load_4d_pair(sm.kv[slot], &tm_k, full_leader, 0, key0 + 32 * static_cast<int>(rank), kv_head, batch);
+          tma_load_4d_pair(sm.kv[slot] + 32 * 64, &tm_k, full_leader, 64, key0 + 32 * static_cast<int>(rank), kv_head,
                            batch);
         } else {
           // all 64 keys, head_dim columns [64 rank, 64 rank + 64)
-          tma_load_4d_pair(S.kv[slot], &tm_v, full_leader, 64 * static_cast<int>(rank), key0, kv_head, batch);
+          tma_load_4d_pair(sm.kv[slot], &tm_v, full_leader, 64 * static_cast<int>(rank), key0, kv_head, batch);
         }
       }
       __syncwarp();
@@ -185,14 +196,14 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // =============================== UMMA issuer (leader CTA) ================================
     if (rank == 0) {
       const uint32_t q_lo0 = umma_desc_lo(smem_u32(S.q[0]), 16);
-      const uint32_t k_lo0 = umma_desc_lo(smem_u32(S.kv[0]), 16);             // as K (K-major)
-      const uint32_t v_lo0 = umma_desc_lo(smem_u32(S.kv[0]), kTileN * 128);   // as V (MN-major, one 64-wide atom)
+      const uint32_t k_lo0 = umma_desc_lo(smem_u32(sm.kv[0]), 16);             // as K (K-major)
+      const uint32_t v_lo0 = umma_desc_lo(smem_u32(sm.kv[0]), kTileN * 128);   // as V (MN-major, one 64-wide atom)
       bool ok = true;
       // S_t = Q K_t^T into S buffer t & 1: eight M256 N64 K16 MMAs
       auto issue_qk = [&](int t) -> bool {
         const int g = 2 * t;
         const int slot = g % kSlots;
-        bool got = mbar_wait(&S.kv_full[slot], (g / kSlots) & 1, &sm.abort_flag, p.status, 41);
+        bool got = mbar_wait(&sm.kv_full[slot], (g / kSlots) & 1, &sm.abort_flag, p.status, 41);
         got = __all_sync(0xffffffffu, got);
         if (!got) return false;
         tc_fence_after();
@@ -221,7 +232,7 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
         const int g = 2 * t + 1;
         const int slot = g % kSlots;
-        ok = mbar_wait2(&S.p_full[t & 1], (t >> 1) & 1, &S.kv_full[slot], (g / kSlots) & 1, &sm.abort_flag, p.status,
+        ok = mbar_wait2(&S.p_full[t & 1], (t >> 1) & 1, &sm.kv_full[slot], (g / kSlots) & 1, &sm.abort_flag, p.status,
                         43);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;

@@ -3,6 +3,9 @@
 // and arrivals in the peer CTA's shared memory, TMA loads that signal a barrier of the peer CTA,
 // tensor-memory allocation for the pair, and UMMA issue / commit for M = 256 tiles.
 //
+// Device status code 4 (beside the codes of sm100_primitives.cuh) = the two CTAs of a pair got different
+// tensor-memory bases and did no work.
+//
 // A kernel uses either these or the cta_group::1 wrappers of sm100_primitives.cuh for its tcgen05
 // allocation, MMA and commit instructions, never both. No load here uses cluster multicast.
 #pragma once
@@ -34,9 +37,12 @@ __device__ __forceinline__ uint32_t ld_cluster_u32(uint32_t cluster_addr) {
   return v;
 }
 
-// One arrival on an mbarrier given by its shared::cluster address (this CTA's or the peer's).
+// One arrival on an mbarrier given by its shared::cluster address (this CTA's or the peer's). Default
+// semantics (release at CTA scope): a cluster-scope release makes the arriving thread wait for all of its earlier
+// global stores, which the callers here neither need nor can afford; what they hand over lives in tensor memory
+// and is ordered by the tcgen05 fences around the arrival.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 // 4-D tiled TMA load into THIS CTA's shared memory whose completion bytes are counted on a barrier
