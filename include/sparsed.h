@@ -146,8 +146,8 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
  * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; the selection needs
  * seq_len / block_size <= 2048 (UNSUPPORTED beyond). Both buffers are caller-owned device memory.
  * sparsed_attn_full_stats runs on a kernel of its own (MMAs spanning pairs of CTAs, launched as
- * clusters of two); the environment variable SPARSED_DENSE_KERNEL=single|pair, read at the first call,
- * sends both dense entry points to one kernel, for measurements.
+ * clusters of two); the environment variable SPARSED_DENSE_KERNEL=pair, read at the first call,
+ * sends sparsed_attn_full to that kernel too, for measurements.
  */
 sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, int32_t block_size,
                                         size_t *out_bytes); /* host only */

@@ -352,18 +352,16 @@ sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stre
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
-// Which dense kernel runs. The pass that also records row statistics goes to the kernel whose MMAs span CTA
-// pairs (its softmax warps have the slack to record them for free: measured 2-5 % faster from 8k to 64k); the
-// plain pass stays on the single-CTA kernel (equal under sustained load, faster on short launches). The
-// environment variable SPARSED_DENSE_KERNEL=pair|single (read once) forces one of them, for A/B measurements.
+// Which dense kernel runs. The pass that also records row statistics has one kernel, whose MMAs span CTA
+// pairs (attention_dense_pair.cu). The plain pass runs the single-CTA kernel (attention.cu: equal under
+// sustained load, faster on short launches) unless the environment says SPARSED_DENSE_KERNEL=pair (read
+// once), which sends it to the pair kernel as well, for A/B measurements and tests.
 static bool dense_pair_kernel(bool with_stats) {
-  static const int forced = [] {
+  static const bool forced = [] {
     const char* v = std::getenv("SPARSED_DENSE_KERNEL");
-    if (v != nullptr && std::strcmp(v, "pair") == 0) return 1;
-    if (v != nullptr && std::strcmp(v, "single") == 0) return 0;
-    return -1;
+    return v != nullptr && std::strcmp(v, "pair") == 0;
   }();
-  return forced >= 0 ? forced == 1 : with_stats;
+  return with_stats || forced;
 }
 
 static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,

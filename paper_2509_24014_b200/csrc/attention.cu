@@ -22,8 +22,8 @@
 //
 // Where the keys come from:
 //   * dense: every 64-key tile of the sequence in order; the last one may be ragged (any seq_len).
-//     Optional outputs: the rows' LSE, and the per-row statistics of each group of 32 / 64 / 128 keys
-//     from which the switch step's pooled scores are formed.
+//     Optional output: the rows' LSE. (The dense pass that also records the row statistics of the switch
+//     step runs on a kernel of its own, attention_dense_pair.cu.)
 //   * 128-key blocks: the 128 query rows are one query block; its CSR list is walked as it is,
 //     two tiles per block.
 //   * 64- and 32-key blocks: the 128 query rows are two / four consecutive query blocks with lists
@@ -32,8 +32,6 @@
 //     its own query block did not keep; a tile in which a warp keeps nothing costs it no
 //     exponentials. All 128 rows of every MMA belong to real queries, and neighbouring query blocks
 //     share the K/V tiles they have in common.
-#include <type_traits>
-
 #include "internal.h"
 #include "softmax_pipeline.cuh"
 
@@ -82,14 +80,12 @@ struct AttnSmem {
 // kDense: walk every key tile of the sequence (kBlock must be 128 then; no block lists are read).
 // kMultiItem: a CTA may be given several query tiles (launched with fewer CTAs than tiles); without it the
 // item loops below run once and their running counters fold to zero at compile time.
-// kStatKeys: dense only: 0, or record one row statistic per 32 / 64 / 128 keys.
-template <int kBlock, bool kDense, bool kMultiItem, int kStatKeys>
+template <int kBlock, bool kDense, bool kMultiItem>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
   static_assert(!kDense || kBlock == 128, "the dense walk uses the unpacked layout");
   static_assert(!kMultiItem || kBlock == 128, "the packed walk prepares its union once per CTA");
-  static_assert(kDense || kStatKeys == 0, "row statistics are recorded by the dense walk only");
   using Smem = AttnSmem<kBlock>;
   constexpr bool kPacked = Smem::kPacked;
   constexpr int kSlots = Smem::kSlots;
@@ -432,20 +428,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int num_tiles = tiles_of(cur);
       const bool group_valid = my_group < cur.groups_here;
       RowState st{-INFINITY, 0.f};
-      RowStatWriter<kStatKeys> stats;
-      if constexpr (kStatKeys > 0) {
-        const int groups = (p.seq_len + kStatKeys - 1) / kStatKeys;
-        float* first = nullptr;
-        if (p.tile_lse != nullptr && cur.q_row0 + tid < p.seq_len)
-          first = p.tile_lse + (static_cast<int64_t>(cur.bh) * p.num_q_tiles + cur.q_tile) * groups * kTileM + tid;
-        stats.init(first, groups);
-      }
-      // One 64-key tile of the softmax. kOdd (a compile-time tag) is only used by the walk that records one
-      // statistic per 128 keys: it runs its tiles in pairs so that the even / odd halves of a statistic are
-      // resolved at compile time instead of costing the busiest warps of the kernel instructions per tile
-      // (pairing every walk was measured too: it costs registers and 2.5 % of the plain dense pass).
-      auto tile_body = [&](int t, auto odd_tag) -> bool {
-        constexpr bool kOdd = decltype(odd_tag)::value;
+      // One 64-key tile of the softmax.
+      auto tile_body = [&](int t) -> bool {
         TL(1);
         // S_t is ready when the Q K^T batch that read ring load 2t of this item has completed
         const int gk = load0 + 2 * t;
@@ -513,7 +497,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             }
           }
           st.l += sums.x + sums.y;
-          if constexpr (kStatKeys > 0) stats.template begin<kOdd>(sums, st.m);
         }
         TL(4);
         tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
@@ -521,17 +504,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tc_fence_before();
         mbar_arrive(&sm.p_full[buf]);
         TL(5);
-        // the statistic is stored after P has been handed over: off the S -> P -> P V chain
-        if constexpr (kStatKeys > 0) stats.template finish<kOdd>(st.m);
         return true;
       };
-      if constexpr (kStatKeys == 128) {
-        int t = 0;
-        for (; ok && t + 1 < num_tiles; t += 2) ok = tile_body(t, std::false_type{}) && tile_body(t + 1, std::true_type{});
-        if (ok && t < num_tiles) ok = tile_body(t, std::false_type{});
-      } else {
-        for (int t = 0; ok && t < num_tiles; ++t) ok = tile_body(t, std::false_type{});
-      }
+      for (int t = 0; ok && t < num_tiles; ++t) ok = tile_body(t);
       if (!ok) break;
 
       // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
@@ -566,10 +541,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   }
 }
 
-template <int kBlock, bool kDense, bool kMultiItem, int kStatKeys>
+template <int kBlock, bool kDense, bool kMultiItem>
 cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
                    int batch, cudaStream_t stream) {
-  auto kernel = attn_kernel<kBlock, kDense, kMultiItem, kStatKeys>;
+  auto kernel = attn_kernel<kBlock, kDense, kMultiItem>;
   const int smem = static_cast<int>(sizeof(AttnSmem<kBlock>));
   static SmemLimit limit;  // per template instantiation
   cudaError_t e = ensure_dynamic_smem(kernel, smem, limit);
@@ -591,18 +566,15 @@ int attn_sparse_max_blocks(int block_size) { return block_size < kTileM ? kMaxPa
 // p.num_q_tiles = ceil(seq_len / 128), p.num_blocks = seq_len / block_size.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128, false, true, 0>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<64, false, false, 0>(tq, tk, tv, p, batch, stream);
-  return launch<32, false, false, 0>(tq, tk, tv, p, batch, stream);
+  if (block_size == 128) return launch<128, false, true>(tq, tk, tv, p, batch, stream);
+  if (block_size == 64) return launch<64, false, false>(tq, tk, tv, p, batch, stream);
+  return launch<32, false, false>(tq, tk, tv, p, batch, stream);
 }
 
 // Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                               const AttnParams& p, int batch, cudaStream_t stream) {
-  if (p.tile_lse == nullptr) return launch<128, true, false, 0>(tq, tk, tv, p, batch, stream);
-  if (p.stat_keys == 128) return launch<128, true, false, 128>(tq, tk, tv, p, batch, stream);
-  if (p.stat_keys == 64) return launch<128, true, false, 64>(tq, tk, tv, p, batch, stream);
-  return launch<128, true, false, 32>(tq, tk, tv, p, batch, stream);
+  return launch<128, true, false>(tq, tk, tv, p, batch, stream);
 }
 
 }  // namespace sparsed

@@ -291,6 +291,7 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
       if (__any_sync(0xffffffffu, exact)) {
         const float alpha = softmax_group_exact(r0, r1, scale_log2, st, pk, sums);
+        if constexpr (kStatKeys > 0) stats.rescale(alpha);
         if (t > 0) {
           // O must be quiescent: wait until P_{t-1} V_{t-1} (which read ring load 2t-1) has drained
           const int gp = 2 * (t - 1) + 1;
@@ -301,14 +302,14 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
       }
       st.l += sums.x + sums.y;
-      if constexpr (kStatKeys > 0) stats.template begin<kOdd>(sums, st.m);
+      if constexpr (kStatKeys > 0) stats.begin(sums, kOdd);
       tmem_st32(tS, pk);  // P_t over the first 32 columns of S_t
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(buf ? p_full_leader1 : p_full_leader0);
       // the statistic is stored after P has been handed over: off the S -> P -> P V chain
-      if constexpr (kStatKeys > 0) stats.template finish<kOdd>(st.m);
+      if constexpr (kStatKeys > 0) stats.finish(st.m, kOdd);
       return true;
     };
     if constexpr (kStatKeys == 128) {

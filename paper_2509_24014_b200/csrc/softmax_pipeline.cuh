@@ -116,8 +116,7 @@ template <int kStatKeys>   // 0 = no statistics, else 32, 64 or 128 keys per sta
 struct RowStatWriter {
   float* next;       // where this row's next statistic goes (statistics of one row are 128 floats apart)
   int left;          // statistics still to be written for this row (0 for rows beyond the sequence end)
-  float carry;       // 128-key groups: sum of the even 64-key half, relative to carry_m
-  float carry_m;
+  float carry;       // 128-key groups: sum of the group's first 64-key half, relative to the CURRENT reference maximum
   float lg0, lg1;    // log2 of the sums of the group in flight (begin -> finish)
 
   // first: the row's first statistic, or null for a row beyond the sequence end; n_groups = ceil(seq_len / kStatKeys)
@@ -125,36 +124,37 @@ struct RowStatWriter {
     next = first;
     left = first != nullptr ? n_groups : 0;
     carry = 0.f;
-    carry_m = 0.f;
     lg0 = lg1 = 0.f;
+  }
+  // The caller's reference maximum moved (exact path): everything summed so far shrinks by alpha = 2^(m_old - m_new).
+  __device__ __forceinline__ void rescale(float alpha) {
+    if constexpr (kStatKeys == 128) carry *= alpha;
   }
   // Two halves, because a warp issues in order: `begin` only STARTS the logarithm(s) as soon as the sums
   // exist; `finish`, called after P has been handed over (by then the results are there), adds the
   // reference maximum and stores. Every instruction here is paid by the softmax warps, the busiest
-  // warps of the kernel (recording costs 5-10 % of the dense pass), hence the running pointer and counter
-  // instead of index arithmetic.
-  // kOdd: this is the second 64-key tile of a 128-key group; sums: the tile's two 32-column sums relative to m.
-  template <bool kOdd>
-  __device__ __forceinline__ void begin(float2 sums, float m) {
+  // warps of the kernel, hence the running pointer and counter instead of index arithmetic, and a carry that
+  // is kept relative to the current maximum (rescaled on the rare exact path) instead of being converted
+  // with an exponential on every second tile.
+  // second_half: 128-key groups only: this is the second 64-key tile of its group; sums: the tile's two
+  // 32-column sums relative to the current reference maximum.
+  __device__ __forceinline__ void begin(float2 sums, bool second_half) {
     if constexpr (kStatKeys == 64) {
       lg0 = fast_log2(sums.x + sums.y);
     } else if constexpr (kStatKeys == 32) {
       lg0 = fast_log2(sums.x);
       lg1 = fast_log2(sums.y);
     } else if constexpr (kStatKeys == 128) {
-      const float s = sums.x + sums.y;
-      if constexpr (!kOdd) {
-        carry = s;
-        carry_m = m;
-      } else {
-        // the even half was summed against carry_m <= m: bring it to the current reference
-        lg0 = fast_log2(fmaf(carry, fast_exp2(carry_m - m), s));
+      carry += sums.x + sums.y;
+      if (second_half) {
+        lg0 = fast_log2(carry);
+        carry = 0.f;
       }
     }
   }
+  // m: the reference maximum the sums given to `begin` were relative to.
   // (a group that lies wholly beyond a ragged sequence end has no statistic: `left` runs out first)
-  template <bool kOdd>
-  __device__ __forceinline__ void finish(float m) {
+  __device__ __forceinline__ void finish(float m, bool second_half) {
     if constexpr (kStatKeys == 64) {
       if (left > 0) __stcs(next, m + lg0);
       next += 128;
@@ -165,7 +165,7 @@ struct RowStatWriter {
       next += 256;
       left -= 2;
     } else if constexpr (kStatKeys == 128) {
-      if constexpr (kOdd) {
+      if (second_half) {
         if (left > 0) __stcs(next, m + lg0);
         next += 128;
         --left;

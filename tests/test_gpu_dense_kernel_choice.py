@@ -1,10 +1,9 @@
-"""Both dense kernels behind both dense entry points.
+"""The CTA-pair dense kernel behind both dense entry points.
 
-By default sparsed_attn_full runs the single-CTA kernel and sparsed_attn_full_stats the kernel whose MMAs span
-CTA pairs; SPARSED_DENSE_KERNEL (read once per process) forces one kernel for both. The oracle parity tests of
-the dense pass and of the statistics path are re-run in child processes with each kernel forced, so that every
-kernel is checked against the oracle through every entry point (ragged lengths, GQA, strided layouts, the
-rescaling path, statistics per 32 / 64 / 128 keys)."""
+sparsed_attn_full_stats always runs the kernel whose MMAs span CTA pairs; sparsed_attn_full runs the single-CTA
+kernel unless SPARSED_DENSE_KERNEL=pair (read once per process). The oracle parity tests of the dense pass are
+re-run in a child process with that setting, so that the pair kernel is also checked on what the statistics
+path never gives it: lengths that are no multiple of 32, strided layouts, a softmax scale, the rescaling path."""
 import os
 import subprocess
 import sys
@@ -15,12 +14,10 @@ pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-@pytest.mark.parametrize("kernel", ["pair", "single"])
-def test_parity_suites_with_forced_dense_kernel(kernel):
-    env = dict(os.environ, SPARSED_DENSE_KERNEL=kernel)
+def test_dense_parity_suite_on_the_pair_kernel():
+    env = dict(os.environ, SPARSED_DENSE_KERNEL="pair")
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
-           "tests/test_gpu_parity_small.py", "tests/test_gpu_switch_step_stats.py", "tests/test_gpu_block32.py",
-           "-k", "attn_full or from_stats or stats or block32_select"]
+           "tests/test_gpu_parity_small.py", "tests/test_gpu_more_cases.py", "-k", "attn_full or entry_point"]
     res = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
     tail = (res.stdout + res.stderr)[-3000:]
     assert res.returncode == 0, tail
