@@ -269,7 +269,7 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // One 64-key tile of the softmax; kOdd (a compile-time tag) is used by the walk that records one statistic per
     // 128 keys, which runs its tiles in pairs.
     auto tile_body = [&](int t, auto odd_tag) -> bool {
-      constexpr bool kOdd = decltype(odd_tag)::value;
+      [[maybe_unused]] constexpr bool kOdd = decltype(odd_tag)::value;
       // S_t is ready when the Q K^T batch that read ring load 2t has completed
       const int gk = 2 * t;
       if (!mbar_wait(&S.done[gk % kSlots], (gk / kSlots) & 1, &sm.abort_flag, p.status, 44)) return false;
