@@ -376,8 +376,9 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
   const bool pair = dense_pair_kernel(tile_lse_or_null != nullptr);
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, to;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&to, o, shape->batch, shape->heads_q, shape->seq_len, rs.o, 128)) != SPARSED_OK) return st;
   if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, pair ? 32 : 64)) != SPARSED_OK) return st;
   if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, 64)) != SPARSED_OK) return st;
   AttnParams p;
@@ -401,8 +402,8 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   p.col_idx = nullptr;
   p.col_capacity = 0;
   p.status = static_cast<DeviceStatus*>(ws);
-  cudaError_t e = pair ? launch_attn_dense_pair(tq, tk, tv, p, static_cast<cudaStream_t>(cuda_stream))
-                      : launch_attn_dense(tq, tk, tv, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = pair ? launch_attn_dense_pair(tq, tk, tv, to, p, static_cast<cudaStream_t>(cuda_stream))
+                      : launch_attn_dense(tq, tk, tv, to, p, shape->batch, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 
@@ -531,8 +532,9 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   if ((st = check_arch()) != SPARSED_OK) return st;
   const int bs = pattern->block_size;
   if (pattern->num_blocks > attn_sparse_max_blocks(bs)) return SPARSED_ERR_UNSUPPORTED;
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, to;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
+  if ((st = make_tensor_map(&to, o, shape->batch, shape->heads_q, shape->seq_len, rs.o, 128)) != SPARSED_OK) return st;
   const int kv_box = bs < 64 ? bs : 64;
   if ((st = make_tensor_map(&tk, k, shape->batch, shape->heads_kv, shape->seq_len, rs.k, kv_box)) != SPARSED_OK) return st;
   if ((st = make_tensor_map(&tv, v, shape->batch, shape->heads_kv, shape->seq_len, rs.v, kv_box)) != SPARSED_OK) return st;
@@ -559,7 +561,7 @@ sparsed_status sparsed_attn_sparse(const sparsed_shape* shape, const sparsed_pat
   p.col_idx = pattern->col_idx;
   p.col_capacity = pattern->col_capacity;
   p.status = static_cast<DeviceStatus*>(ws);
-  cudaError_t e = launch_attn_sparse(tq, tk, tv, p, shape->batch, bs, static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = launch_attn_sparse(tq, tk, tv, to, p, shape->batch, bs, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? SPARSED_OK : cuda_fail(e);
 }
 

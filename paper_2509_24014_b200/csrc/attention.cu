@@ -70,6 +70,7 @@ struct AttnSmem {
   uint64_t q_full, kv_full[kSlots];
   uint64_t done[kSlots];   // the MMAs that read the slot have completed (Q K^T for a K tile, P V for a V tile)
   uint64_t p_full[2];
+  uint64_t q_free;         // an item's output has been read out of the Q buffer (which stages it): the next Q may land
   uint32_t tmem_base;
   int abort_flag;
   int n_union;                                             // packed: key blocks in the union list
@@ -83,7 +84,7 @@ struct AttnSmem {
 template <int kBlock, bool kDense, bool kMultiItem>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-            const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const AttnParams p) {
   static_assert(!kDense || kBlock == 128, "the dense walk uses the unpacked layout");
   static_assert(!kMultiItem || kBlock == 128, "the packed walk prepares its union once per CTA");
   using Smem = AttnSmem<kBlock>;
@@ -203,6 +204,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tma_prefetch_desc(&tm_q);
       tma_prefetch_desc(&tm_k);
       tma_prefetch_desc(&tm_v);
+      if constexpr (!kDense) tma_prefetch_desc(&tm_o);
     }
     __syncwarp();
     if (cur.list_len > 0) {
@@ -220,6 +222,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) mbar_init(&sm.done[s], 1);
     for (int s = 0; s < 2; ++s) mbar_init(&sm.p_full[s], kSoftmaxThreads);
+    mbar_init(&sm.q_free, 1);
     sm.abort_flag = 0;
     sm.n_union = 0;
     mbar_fence_init();
@@ -298,28 +301,37 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     TL_DECL(2)
     bool ok = true;
     int load0 = 0;       // K/V loads issued for earlier items
-    int prev_tiles = 0;  // tiles of the latest earlier item that had any
+    int items_done = 0;  // items before the current one
     for (int item = first_item; ok && item < n_items; item += gridDim.x) {
+      // The Q buffer doubles as the staging tile of the previous item's output: the next Q may land once the
+      // softmax warps have had that output read out of it (which is after the item's last MMA). The first
+      // ring-full of the new item's K/V loads does not depend on its Q (their slots are freed by the previous
+      // item's MMAs), so those go out first and the wait for the Q buffer comes after them. It is waited for in
+      // every item in turn, keys or not, so that this warp is never more than one phase behind the barrier.
+      bool q_pending = false;
       if (item != first_item) {
         cur = describe(item);
-        if (cur.list_len > 0) {
-          if (prev_tiles > 0) {
-            // the Q buffer is free once the previous item's last Q K^T batch (which read load load0 - 2) is done
-            const int g = load0 - 2;
-            ok = mbar_wait(&sm.done[g % kSlots], (g / kSlots) & 1, &sm.abort_flag, p.status, 11);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-          }
-          issue_q_load(cur);
-          if constexpr (!kPacked && !kDense) {
-            list_ids = (lane < cur.list_len) ? __ldg(p.col_idx + cur.list_begin + lane) : 0;
-          }
+        q_pending = true;
+        if constexpr (!kPacked && !kDense) {
+          list_ids = (lane < cur.list_len) ? __ldg(p.col_idx + cur.list_begin + lane) : 0;
         }
       }
+      auto settle_q = [&]() -> bool {
+        bool got = mbar_wait(&sm.q_free, (items_done - 1) & 1, &sm.abort_flag, p.status, 11);
+        got = __all_sync(0xffffffffu, got);
+        if (got && cur.list_len > 0) issue_q_load(cur);
+        q_pending = false;
+        return got;
+      };
       const int n_entries = entries_of(cur);
       const int num_tiles = tiles_of(cur);
+      const int q_at = min(2 * num_tiles, kSlots);
       // load i: K (even) or V (odd) of tile i / 2; a slot is reused every kSlots loads
       for (int i = (item == first_item ? loads_issued : 0); ok && i < 2 * num_tiles; ++i) {
+        if (q_pending && i == q_at && !settle_q()) {
+          ok = false;
+          break;
+        }
         const int t = i >> 1;
         int kv_row0, kv_row1 = 0, blocks_here = 1;
         if constexpr (!kPacked) {
@@ -350,9 +362,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         issue_load(cur, slot, i & 1, kv_row0, kv_row1, blocks_here);
         TL(22);
       }
+      if (ok && q_pending) ok = settle_q();
       if constexpr (!kMultiItem) break;
       load0 += 2 * num_tiles;
-      if (num_tiles > 0) prev_tiles = num_tiles;
+      ++items_done;
     }
   } else if (warp == 5) {
     // =============================== UMMA issuer ========================================
@@ -422,8 +435,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     bool ok = true;
     TL_DECL(0)
     int load0 = 0, tile0 = 0;   // loads / tiles of earlier items
+    [[maybe_unused]] Item nxt = cur;   // multi-item: the next item's row_ptr entries are fetched one item ahead
     for (int item = first_item; ok && item < n_items; item += gridDim.x) {
-      if (item != first_item) cur = describe(item);
+      if constexpr (kMultiItem) {
+        cur = nxt;
+        if (item + static_cast<int>(gridDim.x) < n_items) nxt = describe(item + gridDim.x);
+      }
       const int n_entries = entries_of(cur);
       const int num_tiles = tiles_of(cur);
       const bool group_valid = my_group < cur.groups_here;
@@ -507,23 +524,49 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         return true;
       };
       for (int t = 0; ok && t < num_tiles; ++t) ok = tile_body(t);
-      if (!ok) break;
-
-      // ---- epilogue: O / l -> bf16 -> global (an empty list gives zeros) -------------------
-      if (num_tiles > 0) {
-        const int gl = load0 + 2 * (num_tiles - 1) + 1;   // the last P V read this load's slot
-        ok = mbar_wait(&sm.done[gl % kSlots], (gl / kSlots) & 1, &sm.abort_flag, p.status, 31);
-      }
-      tc_fence_after();
-      const int row = cur.q_row0 + tid;
-      const bool row_valid = row < p.seq_len;
-      const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
-      __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + cur.batch * p.o_stride_b +
-                             cur.head * p.o_stride_h + static_cast<int64_t>(row) * p.o_stride_t;
-      store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
       if constexpr (kDense) {
+        // ---- epilogue of the dense walk: O / l -> bf16 -> global, each row from its own thread ----------
+        // (with the staged epilogue of the other walks its main loop compiled 1-2 % slower, measured, and its
+        // epilogue is 0.3 % of a 64k launch)
+        if (!ok) break;
+        if (num_tiles > 0) {
+          const int gl = load0 + 2 * (num_tiles - 1) + 1;   // the last P V read this load's slot
+          ok = mbar_wait(&sm.done[gl % kSlots], (gl / kSlots) & 1, &sm.abort_flag, p.status, 31);
+        }
+        tc_fence_after();
+        const int row = cur.q_row0 + tid;
+        const bool row_valid = row < p.seq_len;
+        const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
+        __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + cur.batch * p.o_stride_b +
+                               cur.head * p.o_stride_h + static_cast<int64_t>(row) * p.o_stride_t;
+        store_output_row(tO + lane_base, num_tiles > 0, inv_l, o_row, row_valid);
         if (p.lse != nullptr && row_valid)
           p.lse[static_cast<int64_t>(cur.bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
+      } else {
+        // ---- epilogue: O / l -> bf16 -> shared memory -> global (an empty list gives zeros) ----------
+        // Every thread goes through the barrier below even after a wait has run out (it then stages zeros), so
+        // that none is left waiting there; what is done after it is decided by the shared flag.
+        if (ok && num_tiles > 0) {
+          const int gl = load0 + 2 * (num_tiles - 1) + 1;   // the last P V read this load's slot
+          ok = mbar_wait(&sm.done[gl % kSlots], (gl / kSlots) & 1, &sm.abort_flag, p.status, 31);
+        }
+        tc_fence_after();
+        const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
+        // The Q tile is dead (the item's last Q K^T completed before its last P V did): it stages the output
+        // tile. After an item without keys nothing made these threads wait for the previous tile to be read out:
+        // they meet the thread that waited for that here.
+        if (num_tiles == 0) named_barrier_sync(1, kSoftmaxThreads);
+        stage_output_row(tO + lane_base, ok && num_tiles > 0, inv_l, &sm.q[0][0], tid);
+        named_barrier_sync(1, kSoftmaxThreads);
+        if (*reinterpret_cast<volatile int*>(&sm.abort_flag) != 0) break;
+        if (tid == 0) {
+          // rows beyond the sequence end are clipped by the tensor map
+          tma_store_4d(&tm_o, sm.q[0], 0, cur.q_row0, cur.head, cur.batch);
+          tma_store_4d(&tm_o, sm.q[1], 64, cur.q_row0, cur.head, cur.batch);
+          tma_store_commit();
+          tma_store_wait_read();
+          if constexpr (kMultiItem) mbar_arrive(&sm.q_free);
+        }
       }
       if constexpr (!kMultiItem) break;
       tc_fence_before();   // the next item's first P V overwrites O: order these reads before its hand-over
@@ -542,8 +585,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 }
 
 template <int kBlock, bool kDense, bool kMultiItem>
-cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
-                   int batch, cudaStream_t stream) {
+cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                   const AttnParams& p, int batch, cudaStream_t stream) {
   auto kernel = attn_kernel<kBlock, kDense, kMultiItem>;
   const int smem = static_cast<int>(sizeof(AttnSmem<kBlock>));
   static SmemLimit limit;  // per template instantiation
@@ -554,7 +597,7 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
   long long ctas = p.num_items;
   if (ctas <= 0) return cudaSuccess;
   if (kMultiItem && p.max_ctas > 0 && ctas > p.max_ctas) ctas = p.max_ctas;
-  kernel<<<static_cast<unsigned>(ctas), kThreads, smem, stream>>>(tq, tk, tv, p);
+  kernel<<<static_cast<unsigned>(ctas), kThreads, smem, stream>>>(tq, tk, tv, to, p);
   return cudaGetLastError();
 }
 
@@ -562,19 +605,20 @@ cudaError_t launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
 
 int attn_sparse_max_blocks(int block_size) { return block_size < kTileM ? kMaxPackedBlocks : 16384; }
 
-// Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x min(64, block_size) rows.
+// Tensor maps: Q and O boxes 64 x 128 rows, K and V boxes 64 x min(64, block_size) rows.
 // p.num_q_tiles = ceil(seq_len / 128), p.num_blocks = seq_len / block_size.
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                               const AttnParams& p, int batch, int block_size, cudaStream_t stream) {
-  if (block_size == 128) return launch<128, false, true>(tq, tk, tv, p, batch, stream);
-  if (block_size == 64) return launch<64, false, false>(tq, tk, tv, p, batch, stream);
-  return launch<32, false, false>(tq, tk, tv, p, batch, stream);
+                               const CUtensorMap& to, const AttnParams& p, int batch, int block_size,
+                               cudaStream_t stream) {
+  if (block_size == 128) return launch<128, false, true>(tq, tk, tv, to, p, batch, stream);
+  if (block_size == 64) return launch<64, false, false>(tq, tk, tv, to, p, batch, stream);
+  return launch<32, false, false>(tq, tk, tv, to, p, batch, stream);
 }
 
-// Tensor maps: Q box 64 x 128 rows, K and V boxes 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
+// Tensor maps: Q and O boxes 64 x 128 rows, K and V boxes 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                              const AttnParams& p, int batch, cudaStream_t stream) {
-  return launch<128, true, false>(tq, tk, tv, p, batch, stream);
+                              const CUtensorMap& to, const AttnParams& p, int batch, cudaStream_t stream) {
+  return launch<128, true, false>(tq, tk, tv, to, p, batch, stream);
 }
 
 }  // namespace sparsed

@@ -71,7 +71,8 @@ constexpr uint32_t kSlotStep = (kTileN * 64 * 2) >> 4;                   // 8 KB
 template <int kStatKeys>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                       const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   PairSmem& sm = *reinterpret_cast<PairSmem*>(smem_raw);
   const int tid = threadIdx.x;
@@ -113,6 +114,7 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tma_prefetch_desc(&tm_q);
     tma_prefetch_desc(&tm_k);
     tma_prefetch_desc(&tm_v);
+    tma_prefetch_desc(&tm_o);
   }
   if (warp == 10) {
     tmem_alloc_pair(&sm.tmem_base, kTmemCols);
@@ -319,21 +321,29 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     } else {
       for (int t = 0; ok && t < num_tiles; ++t) ok = tile_body(t, std::false_type{});
     }
+    // ---- epilogue: O / l -> bf16 -> shared memory -> global -----------------------------------
+    // Every thread goes through the barrier below even after a wait has run out (it then stages zeros), so that
+    // none is left waiting there; what is done after it is decided by the shared flag.
     if (ok) {
-      // ---- epilogue: O / l -> bf16 -> global ---------------------------------------------
       const int gl = 2 * (num_tiles - 1) + 1;   // the last P V read this load's slot
       ok = mbar_wait(&S.done[gl % kSlots], (gl / kSlots) & 1, &sm.abort_flag, p.status, 46);
-      tc_fence_after();
-      if (ok) {
-        const int row = q_row0 + row_in_tile;
-        const bool row_valid = row < p.seq_len;
-        const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
-        __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + batch * p.o_stride_b + head * p.o_stride_h +
-                               static_cast<int64_t>(row) * p.o_stride_t;
-        store_output_row(tO + lane_base, true, inv_l, o_row, row_valid);
-        if (p.lse != nullptr && row_valid)
-          p.lse[static_cast<int64_t>(bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
+    }
+    tc_fence_after();
+    const int row = q_row0 + row_in_tile;
+    const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
+    // the stream's Q tile is dead (its last Q K^T completed before its last P V did): it stages the output tile
+    stage_output_row(tO + lane_base, ok, inv_l, &S.q[0][0], row_in_tile);
+    named_barrier_sync(1 + s_of_warp, kTileM);
+    if (*reinterpret_cast<volatile int*>(&sm.abort_flag) == 0) {
+      if (row_in_tile == 0 && q_row0 < p.seq_len) {
+        // rows beyond the sequence end are clipped by the tensor map
+        tma_store_4d(&tm_o, S.q[0], 0, q_row0, head, batch);
+        tma_store_4d(&tm_o, S.q[1], 64, q_row0, head, batch);
+        tma_store_commit();
+        tma_store_wait_read();
       }
+      if (p.lse != nullptr && row < p.seq_len)
+        p.lse[static_cast<int64_t>(bh) * p.seq_len + row] = (st.m + log2f(st.l)) * 0.69314718055994531f;
     }
   }
 
@@ -350,8 +360,8 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 }
 
 template <int kStatKeys>
-cudaError_t launch_pair(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& p,
-                        cudaStream_t stream) {
+cudaError_t launch_pair(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                        const AttnParams& p, cudaStream_t stream) {
   auto kernel = attn_dense_pair_kernel<kStatKeys>;
   const int smem = static_cast<int>(sizeof(PairSmem));
   static SmemLimit limit;  // per template instantiation
@@ -360,19 +370,19 @@ cudaError_t launch_pair(const CUtensorMap& tq, const CUtensorMap& tk, const CUte
   const long long bh = p.num_q_tiles > 0 ? p.num_items / p.num_q_tiles : 0;
   const long long clusters = bh * ((p.num_q_tiles + 3) / 4);
   if (clusters <= 0) return cudaSuccess;
-  kernel<<<static_cast<unsigned>(2 * clusters), kThreads, smem, stream>>>(tq, tk, tv, p);
+  kernel<<<static_cast<unsigned>(2 * clusters), kThreads, smem, stream>>>(tq, tk, tv, to, p);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-// Tensor maps: Q box 64 x 128 rows, K box 64 x 32 rows, V box 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
+// Tensor maps: Q and O boxes 64 x 128 rows, K box 64 x 32 rows, V box 64 x 64 rows. p.num_q_tiles = ceil(seq_len / 128).
 cudaError_t launch_attn_dense_pair(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                   const AttnParams& p, cudaStream_t stream) {
-  if (p.tile_lse == nullptr) return launch_pair<0>(tq, tk, tv, p, stream);
-  if (p.stat_keys == 128) return launch_pair<128>(tq, tk, tv, p, stream);
-  if (p.stat_keys == 64) return launch_pair<64>(tq, tk, tv, p, stream);
-  return launch_pair<32>(tq, tk, tv, p, stream);
+                                   const CUtensorMap& to, const AttnParams& p, cudaStream_t stream) {
+  if (p.tile_lse == nullptr) return launch_pair<0>(tq, tk, tv, to, p, stream);
+  if (p.stat_keys == 128) return launch_pair<128>(tq, tk, tv, to, p, stream);
+  if (p.stat_keys == 64) return launch_pair<64>(tq, tk, tv, to, p, stream);
+  return launch_pair<32>(tq, tk, tv, to, p, stream);
 }
 
 }  // namespace sparsed

@@ -36,7 +36,8 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, SmemLimit& lim)
 
 // Parameters shared by the dense and the block-sparse attention kernels.
 struct AttnParams {
-  void* o;                 // bf16 [B,Hq,L,D]
+  void* o;                 // bf16 [B,Hq,L,D]; used by the plain dense kernel, which stores rows itself (the others
+                           // write O through its tensor map)
   int64_t o_stride_b, o_stride_h, o_stride_t;
   float* lse;              // fp32 [B,Hq,L] or null
   float* tile_lse;         // fp32 [B*Hq, ceil(L/128), ceil(L/stat_keys), 128] or null: base-2 log-sum-exp of each row over each group of stat_keys keys
@@ -119,14 +120,16 @@ constexpr int kPooledQkMaxBlocks = 1024;
 
 size_t pooled_qk_means_bytes(int batch, int heads_q, int heads_kv, int nb);
 cudaError_t launch_pooled_qk_select(const PooledQkParams& p, cudaStream_t stream);
+// (`to`: tensor map of the output, boxes of 64 x 128 rows like Q's; the kernels write O through it)
 cudaError_t launch_attn_dense(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                              const AttnParams& p, int batch, cudaStream_t stream);
+                              const CUtensorMap& to, const AttnParams& p, int batch, cudaStream_t stream);
 // The same pass with the MMAs spanning CTA pairs (cta_group::2); K tensor map with 32-row boxes.
 cudaError_t launch_attn_dense_pair(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                   const AttnParams& p, cudaStream_t stream);
+                                   const CUtensorMap& to, const AttnParams& p, cudaStream_t stream);
 int attn_sparse_max_blocks(int block_size);   // most key blocks per row the sparse kernel handles
 cudaError_t launch_attn_sparse(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                               const AttnParams& p, int batch, int block_size, cudaStream_t stream);
+                               const CUtensorMap& to, const AttnParams& p, int batch, int block_size,
+                               cudaStream_t stream);
 cudaError_t launch_row_stats(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, float* lse_out,
                              int batch, cudaStream_t stream);
 cudaError_t launch_pooled_scores(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int batch,
