@@ -70,7 +70,7 @@ struct AttnSmem {
   uint64_t q_full, kv_full[kSlots];
   uint64_t done[kSlots];   // the MMAs that read the slot have completed (Q K^T for a K tile, P V for a V tile)
   uint64_t p_full[2];
-  uint64_t q_free;         // an item's output has been read out of the Q buffer (which stages it): the next Q may land
+  uint64_t q_free;         // an output tile has been read out of the Q buffer (which staged it): the next Q may land
   uint32_t tmem_base;
   int abort_flag;
   int n_union;                                             // packed: key blocks in the union list
@@ -301,25 +301,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     TL_DECL(2)
     bool ok = true;
     int load0 = 0;       // K/V loads issued for earlier items
-    int items_done = 0;  // items before the current one
+    int q_tiles_done = 0;  // earlier items that had keys (each loaded a Q tile and staged an output tile)
     for (int item = first_item; ok && item < n_items; item += gridDim.x) {
-      // The Q buffer doubles as the staging tile of the previous item's output: the next Q may land once the
-      // softmax warps have had that output read out of it (which is after the item's last MMA). The first
-      // ring-full of the new item's K/V loads does not depend on its Q (their slots are freed by the previous
-      // item's MMAs), so those go out first and the wait for the Q buffer comes after them. It is waited for in
-      // every item in turn, keys or not, so that this warp is never more than one phase behind the barrier.
+      // The Q buffer doubles as the staging tile of the previous output: the next Q may land once the softmax
+      // warps have had that output read out of it (which is after the item's last MMA). The first ring-full of
+      // the new item's K/V loads does not depend on its Q (their slots are freed by the previous item's MMAs),
+      // so those go out first and the wait for the Q buffer comes after them. Items without keys take no part
+      // in this (no Q tile, zeros stored straight from registers), so the barrier completes exactly once per Q
+      // tile and this warp is never more than one phase away from it.
       bool q_pending = false;
       if (item != first_item) {
         cur = describe(item);
-        q_pending = true;
+        q_pending = cur.list_len > 0;
         if constexpr (!kPacked && !kDense) {
           list_ids = (lane < cur.list_len) ? __ldg(p.col_idx + cur.list_begin + lane) : 0;
         }
       }
       auto settle_q = [&]() -> bool {
-        bool got = mbar_wait(&sm.q_free, (items_done - 1) & 1, &sm.abort_flag, p.status, 11);
-        got = __all_sync(0xffffffffu, got);
-        if (got && cur.list_len > 0) issue_q_load(cur);
+        bool got = true;
+        if (q_tiles_done > 0) {
+          got = mbar_wait(&sm.q_free, (q_tiles_done - 1) & 1, &sm.abort_flag, p.status, 11);
+          got = __all_sync(0xffffffffu, got);
+        }
+        if (got) issue_q_load(cur);
         q_pending = false;
         return got;
       };
@@ -365,7 +369,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (ok && q_pending) ok = settle_q();
       if constexpr (!kMultiItem) break;
       load0 += 2 * num_tiles;
-      ++items_done;
+      if (num_tiles > 0) ++q_tiles_done;
     }
   } else if (warp == 5) {
     // =============================== UMMA issuer ========================================
@@ -552,20 +556,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         tc_fence_after();
         const float inv_l = st.l > 0.f ? (1.f / st.l) : 0.f;
-        // The Q tile is dead (the item's last Q K^T completed before its last P V did): it stages the output
-        // tile. After an item without keys nothing made these threads wait for the previous tile to be read out:
-        // they meet the thread that waited for that here.
-        if (num_tiles == 0) named_barrier_sync(1, kSoftmaxThreads);
-        stage_output_row(tO + lane_base, ok && num_tiles > 0, inv_l, &sm.q[0][0], tid);
-        named_barrier_sync(1, kSoftmaxThreads);
-        if (*reinterpret_cast<volatile int*>(&sm.abort_flag) != 0) break;
-        if (tid == 0) {
-          // rows beyond the sequence end are clipped by the tensor map
-          tma_store_4d(&tm_o, sm.q[0], 0, cur.q_row0, cur.head, cur.batch);
-          tma_store_4d(&tm_o, sm.q[1], 64, cur.q_row0, cur.head, cur.batch);
-          tma_store_commit();
-          tma_store_wait_read();
-          if constexpr (kMultiItem) mbar_arrive(&sm.q_free);
+        if (num_tiles == 0) {
+          // no keys: zeros, straight from registers (the Q buffer may already hold a later item's tile)
+          const int row = cur.q_row0 + tid;
+          __nv_bfloat16* o_row = reinterpret_cast<__nv_bfloat16*>(p.o) + cur.batch * p.o_stride_b +
+                                 cur.head * p.o_stride_h + static_cast<int64_t>(row) * p.o_stride_t;
+          store_output_row(0u, false, 0.f, o_row, row < p.seq_len);
+        } else {
+          // The Q tile is dead (the item's last Q K^T completed before its last P V did): it stages the output.
+          stage_output_row(tO + lane_base, ok, inv_l, &sm.q[0][0], tid);
+          named_barrier_sync(1, kSoftmaxThreads);
+          if (*reinterpret_cast<volatile int*>(&sm.abort_flag) != 0) break;
+          if (tid == 0) {
+            // rows beyond the sequence end are clipped by the tensor map
+            tma_store_4d(&tm_o, sm.q[0], 0, cur.q_row0, cur.head, cur.batch);
+            tma_store_4d(&tm_o, sm.q[1], 64, cur.q_row0, cur.head, cur.batch);
+            tma_store_commit();
+            tma_store_wait_read();
+            if constexpr (kMultiItem) mbar_arrive(&sm.q_free);
+          }
         }
       }
       if constexpr (!kMultiItem) break;

@@ -184,7 +184,7 @@ def test_token_major_layout_through_every_entry_point():
 def test_ctas_that_run_through_several_query_tiles_match_one_tile_per_cta():
     """Block-sparse launches with more query tiles than CTAs fit on the device let every CTA roll on into
     further tiles (ring slots, S buffers and barrier phases carry over). 768 query tiles with ragged
-    user-built lists, empty ones among them, must give bitwise what the same heads give when launched one
+    user-built lists, single empty ones and runs of them among them, must give bitwise what the same heads give when launched one
     head at a time (64 tiles each: one tile per CTA), and agree with the oracle on sampled rows."""
     B, Hq, Hkv, L, bs = 1, 12, 4, 8192, 128
     cfg = syn.AttnConfig("roll", B, Hq, Hkv, L, 128, bs, 0.1, 0, seed=404, plant_norm=6.0)
@@ -193,7 +193,8 @@ def test_ctas_that_run_through_several_query_tiles_match_one_tile_per_cta():
     rng = np.random.default_rng(404)
     lists = []
     for r in range(Hq * nb):
-        n = int(rng.integers(0, 7)) if r % 5 else 0             # every fifth list is empty
+        # every fifth list is empty, and so is a run of six neighbouring ones in every head
+        n = int(rng.integers(0, 7)) if (r % 5 and not 40 <= r % 64 < 46) else 0
         lists.append(sorted(rng.choice(nb, size=n, replace=False).tolist()))
     rp = np.cumsum([0] + [len(x) for x in lists]).astype(np.int32)
     ci = np.concatenate([np.asarray(x, dtype=np.int32) for x in lists] + [np.zeros(1, np.int32)]).astype(np.int32)
@@ -211,7 +212,7 @@ def test_ctas_that_run_through_several_query_tiles_match_one_tile_per_cta():
     torch.cuda.synchronize()
     assert sd.sparsed_last_device_status(ws) == (0, 0)
     assert torch.equal(o_all, o_one)
-    for h, ib in ((0, 0), (3, 17), (7, 63), (11, 40), (5, 5)):
+    for h, ib in ((0, 0), (3, 17), (7, 63), (11, 40), (5, 5), (2, 43), (9, 46)):
         r = h * nb + ib
         rows = slice(ib * bs, (ib + 1) * bs)
         if not lists[r]:
