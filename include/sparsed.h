@@ -17,6 +17,8 @@
  *    The fp32 side buffers (lse, tile_stats, scores, scores_out) and the workspace must be
  *    16-byte aligned too (the kernels read them with 16-byte loads), row_ptr and col_idx
  *    4-byte aligned; anything else is refused with SPARSED_ERR_ALIGNMENT before any launch.
+ *    Output buffers (O, lse, tile_stats, scores_out, the pattern arrays) must not overlap any
+ *    input of the same call: the kernels write them while other thread blocks still read.
  *  - Grouped-query attention: query head h reads key/value head h / (heads_q / heads_kv).
  *  - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *    stream) and return without synchronising. Argument problems are detected on the
