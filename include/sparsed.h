@@ -147,9 +147,10 @@ sparsed_status sparsed_select_from_scores(const sparsed_select_params *params, c
  *                               recorded with.
  * Same rules and errors as sparsed_attn_full / sparsed_select_pattern; the selection needs
  * seq_len / block_size <= 2048 (UNSUPPORTED beyond). Both buffers are caller-owned device memory.
- * sparsed_attn_full_stats runs on a kernel of its own (MMAs spanning pairs of CTAs, launched as
- * clusters of two); the environment variable SPARSED_DENSE_KERNEL=pair, read at the first call,
- * sends sparsed_attn_full to that kernel too, for measurements.
+ * sparsed_attn_full_stats runs on a kernel whose MMAs span pairs of CTAs (launched as clusters of two);
+ * sparsed_attn_full runs on it from 16384 tokens on and on a single-CTA kernel below that. The environment
+ * variable SPARSED_DENSE_KERNEL=pair|single, read at the first call, sends sparsed_attn_full to one of
+ * them at every length, for measurements.
  */
 sparsed_status sparsed_tile_stats_bytes(const sparsed_shape *shape, int32_t block_size,
                                         size_t *out_bytes); /* host only */

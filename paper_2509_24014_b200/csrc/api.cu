@@ -353,15 +353,19 @@ sparsed_status sparsed_workspace_init(void* ws, size_t ws_bytes, void* cuda_stre
 }
 
 // Which dense kernel runs. The pass that also records row statistics has one kernel, whose MMAs span CTA
-// pairs (attention_dense_pair.cu). The plain pass runs the single-CTA kernel (attention.cu: equal under
-// sustained load, faster on short launches) unless the environment says SPARSED_DENSE_KERNEL=pair (read
-// once), which sends it to the pair kernel as well, for A/B measurements and tests.
-static bool dense_pair_kernel(bool with_stats) {
-  static const bool forced = [] {
+// pairs (attention_dense_pair.cu). The plain pass runs it from 16k tokens on (measured 3-4 % faster there) and
+// the single-CTA kernel (attention.cu) below that, where a cluster's short life makes the pair kernel no
+// faster under sustained load and slower per launch. The environment variable SPARSED_DENSE_KERNEL (read once)
+// sends every plain pass to one of them, `pair` or `single`, for A/B measurements and tests.
+static bool dense_pair_kernel(bool with_stats, int seq_len) {
+  static const int forced = [] {
     const char* v = std::getenv("SPARSED_DENSE_KERNEL");
-    return v != nullptr && std::strcmp(v, "pair") == 0;
+    if (v != nullptr && std::strcmp(v, "pair") == 0) return 1;
+    if (v != nullptr && std::strcmp(v, "single") == 0) return 0;
+    return -1;
   }();
-  return with_stats || forced;
+  if (with_stats) return true;
+  return forced >= 0 ? forced == 1 : seq_len >= 16384;
 }
 
 static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, const void* k, const void* v, void* o,
@@ -375,7 +379,7 @@ static sparsed_status attn_full_impl(const sparsed_shape* shape, const void* q, 
   if (!aligned16(lse_or_null) || !aligned16(tile_lse_or_null)) return SPARSED_ERR_ALIGNMENT;
   if ((st = check_ws(ws, ws_bytes, SPARSED_STATUS_BYTES)) != SPARSED_OK) return st;
   if ((st = check_arch()) != SPARSED_OK) return st;
-  const bool pair = dense_pair_kernel(tile_lse_or_null != nullptr);
+  const bool pair = dense_pair_kernel(tile_lse_or_null != nullptr, shape->seq_len);
   CUtensorMap tq, tk, tv, to;
   if ((st = make_tensor_map(&tq, q, shape->batch, shape->heads_q, shape->seq_len, rs.q, 128)) != SPARSED_OK) return st;
   if ((st = make_tensor_map(&to, o, shape->batch, shape->heads_q, shape->seq_len, rs.o, 128)) != SPARSED_OK) return st;

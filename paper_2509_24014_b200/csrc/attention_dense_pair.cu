@@ -314,12 +314,10 @@ attn_dense_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if constexpr (kStatKeys > 0) stats.finish(st.m, kOdd);
       return true;
     };
-    if constexpr (kStatKeys == 128) {
+    {
       int t = 0;
       for (; ok && t + 1 < num_tiles; t += 2) ok = tile_body(t, std::false_type{}) && tile_body(t + 1, std::true_type{});
       if (ok && t < num_tiles) ok = tile_body(t, std::false_type{});
-    } else {
-      for (int t = 0; ok && t < num_tiles; ++t) ok = tile_body(t, std::false_type{});
     }
     // ---- epilogue: O / l -> bf16 -> shared memory -> global -----------------------------------
     // Every thread goes through the barrier below even after a wait has run out (it then stages zeros), so that
