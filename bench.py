@@ -49,20 +49,20 @@ _ATTN_SHA = "70443f629121"
 _PAIR_SRC = ("paper_2509_24014_b200/csrc/attention_dense_pair.cu", "paper_2509_24014_b200/csrc/sm100_pair_primitives.cuh",
              "paper_2509_24014_b200/csrc/softmax_pipeline.cuh", "paper_2509_24014_b200/csrc/sm100_primitives.cuh",
              "paper_2509_24014_b200/build.py")   # (its compile flags are set per file there)
-_PAIR_SHA = "d50fa104bc60"
+_PAIR_SHA = "6d0bd09b545c"
 _POOL_SRC = ("paper_2509_24014_b200/csrc/pool_select.cu", "paper_2509_24014_b200/csrc/topk_device.cuh")
 _POOL_SHA = "2a48dbebbbc2"
 NCU_DRAM_TRAFFIC = {
-    ("attn_dense_pair_kernel", "c2"): (201653504 + 103153408, _C2_ATTN, _PAIR_SRC, _PAIR_SHA),
-    ("attn_kernel<sparse>", "c2"): (156463616 + 44160768, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
+    ("attn_dense_pair_kernel", "c2"): (201576192 + 102648320, _C2_ATTN, _PAIR_SRC, _PAIR_SHA),
+    ("attn_kernel<sparse>", "c2"): (156466176 + 43784192, _C2_ATTN, _ATTN_SRC, _ATTN_SHA),
     ("pool_select_kernel", "c2"): (68194816 + 587776, _C2_POOL, _POOL_SRC, _POOL_SHA),
     # 64k workload: the 8k capture scaled by the algorithmic bytes of a launch (traffic was the algorithmic
     # traffic at 8k: every K/V re-read hits L2), instead of a multi-counter capture of a 7 GB workload.
     # dense + statistics: Q,K,V,O + LSE + statistics = 6450 MB at 64k against 336 MB at 8k
-    ("attn_dense_pair_kernel", "c4"): (int((201653504 + 103153408) * 6450.0 / 336.0), _C2_ATTN + ", scaled x19.2 by algorithmic bytes",
+    ("attn_dense_pair_kernel", "c4"): (int((201576192 + 102648320) * 6450.0 / 336.0), _C2_ATTN + ", scaled x19.2 by algorithmic bytes",
                                        _PAIR_SRC, _PAIR_SHA),
     # sparse: Q + O + touched K,V: 8x the rows and 8x the K/V of the 8k workload
-    ("attn_kernel<sparse>", "c4"): ((156463616 + 44160768) * 8, _C2_ATTN + ", scaled x8 by algorithmic bytes",
+    ("attn_kernel<sparse>", "c4"): ((156466176 + 43784192) * 8, _C2_ATTN + ", scaled x8 by algorithmic bytes",
                                     _ATTN_SRC, _ATTN_SHA),
     # pooling: the statistics stream, 64x the 8k one (rows x8, key blocks x8)
     ("pool_select_kernel", "c4"): ((68194816 + 587776) * 64, _C2_POOL + ", scaled x64 by algorithmic bytes",
