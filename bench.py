@@ -45,11 +45,11 @@ _C2_ATTN = "ncu --set full capture of one launch on the 8k workload (summary und
 _C2_POOL = "ncu --set full capture of one launch on the 8k workload (summary under profiles/)"
 _ATTN_SRC = ("paper_2509_24014_b200/csrc/attention.cu", "paper_2509_24014_b200/csrc/softmax_pipeline.cuh",
              "paper_2509_24014_b200/csrc/sm100_primitives.cuh")
-_ATTN_SHA = "70443f629121"
+_ATTN_SHA = "258d6b93c29d"
 _PAIR_SRC = ("paper_2509_24014_b200/csrc/attention_dense_pair.cu", "paper_2509_24014_b200/csrc/sm100_pair_primitives.cuh",
              "paper_2509_24014_b200/csrc/softmax_pipeline.cuh", "paper_2509_24014_b200/csrc/sm100_primitives.cuh",
              "paper_2509_24014_b200/build.py")   # (its compile flags are set per file there)
-_PAIR_SHA = "6d0bd09b545c"
+_PAIR_SHA = "ac9c2ae83227"
 _POOL_SRC = ("paper_2509_24014_b200/csrc/pool_select.cu", "paper_2509_24014_b200/csrc/topk_device.cuh")
 _POOL_SHA = "2a48dbebbbc2"
 NCU_DRAM_TRAFFIC = {

@@ -7,7 +7,7 @@
 // tensor-memory bases and did no work.
 //
 // A kernel uses either these or the cta_group::1 wrappers of sm100_primitives.cuh for its tcgen05
-// allocation, MMA and commit instructions, never both. No load here uses cluster multicast.
+// allocation, MMA and commit instructions, never both. Every CTA loads its own tiles: no load here delivers to more than one CTA.
 #pragma once
 
 #include "sm100_primitives.cuh"
@@ -46,7 +46,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
 }
 
 // 4-D tiled TMA load into THIS CTA's shared memory whose completion bytes are counted on a barrier
-// that may live in the peer CTA (given as a shared::cluster address). No multicast.
+// that may live in the peer CTA (given as a shared::cluster address); the data go to this CTA alone.
 // Coordinates are innermost first; c0 * sizeof(element) must be a multiple of 16.
 __device__ __forceinline__ void tma_load_4d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr, int c0,
                                                  int c1, int c2, int c3) {

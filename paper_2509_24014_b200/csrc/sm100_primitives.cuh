@@ -120,7 +120,7 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 }
 
 // ----------------------------------------------------------------------------
-// TMA (cp.async.bulk.tensor), 4-D tiled load, no multicast.
+// TMA: 4-D tiled load into the issuing CTA's own shared memory (every CTA loads for itself).
 // Coordinates are innermost first.  c0 * sizeof(element) must be a multiple of 16.
 // ----------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, uint64_t* bar, int c0, int c1,
